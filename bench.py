@@ -1,0 +1,330 @@
+#!/usr/bin/env python
+"""Benchmark of the HiViS drafter step (draft steps/s, us/step, HBM roofline fraction).
+
+One benchmark "step" = one pass of the hot path over one batch: k chained draft steps
+(fuse+residual, RMSNorm, QKV, RoPE, attention over the text-only cache, O, SwiGLU, LM head,
+argmax) followed by batched greedy verification with KV rollback.  `value` counts draft steps
+(k per benchmark step).  Inputs are seeded and synthetic; weights are random-init in the shape of
+the named backbone.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import hivis_inputs as hi  # noqa: E402
+
+METRIC = "draft_steps_per_s"
+UNIT = "draft steps/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu, self.rows, self.proc = gpu_index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], None, set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[1])); mx = float(r[2])
+            except Exception:
+                continue
+            for name, col in (("hw_slowdown", 5), ("hw_thermal_slowdown", 6), ("sw_thermal_slowdown", 7),
+                              ("sw_power_cap", 8)):
+                if len(r) > col and r[col].lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def run_oracle_sample(wl, steps: int, warmup: int):
+    """The CPU oracle (fp32 build) as it stands, timed on the host cores on a bounded sample of
+    the same workload: the k-step chain of the first sequence(s) after an untimed prefill."""
+    import oracle
+    W = hi.make_weights(wl.dims, wl.seed)
+    ids, hidden, cu = hi.make_prompt(wl)
+    resid = hi.make_residuals(wl)
+    o = oracle.Oracle(wl.dims, W, "f32")
+    rho = o.fold_residuals(resid)
+    nseq = min(wl.batch, 2)
+    caches = []
+    for b in range(nseq):
+        lo, hi_ = int(cu[b]), int(cu[b + 1])
+        T = hi_ - lo
+        Kc, Vc = o.new_cache(T + wl.k)
+        o.prefill(ids[lo:hi_], hidden[lo:hi_], rho[0], Kc, Vc)
+        caches.append((T, Kc, Vc, int(ids[hi_ - 1]), hidden[hi_ - 1]))
+    times = []
+    for it in range(warmup + steps):
+        t0 = time.perf_counter()
+        for (T, Kc, Vc, pid, ph) in caches:
+            o.draft(T - 1, pid, ph, wl.k, rho, Kc, Vc, want_logits=False)
+        times.append(time.perf_counter() - t0)
+    t = float(np.mean(times[warmup:]))
+    per_seq_step = t / (nseq * wl.k)
+    # one batched draft step on the CPU = batch sequential single-sequence steps
+    return {"value": 1.0 / (per_seq_step * wl.batch), "unit": UNIT, "cores": o.num_threads(), "kind": "oracle",
+            "sample": f"{steps} timed repetitions (after {warmup} warm-up) of the {wl.k}-step chain for {nseq} of "
+                      f"{wl.batch} sequence(s), prefill untimed; a batched step costed as batch x the "
+                      f"single-sequence step", "us_per_step": per_seq_step * wl.batch * 1e6,
+            "ms_per_bench_step": t / nseq * wl.batch * 1e3}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2_llava_b1")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    wl = hi.workload(args.workload)
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    config = {"workload": wl.name, "batch": wl.batch, "k": wl.k, "draft_steps_per_bench_step": wl.k,
+              "text_len": wl.text_len if wl.text_len else list(wl.text_len_range),
+              "leading_positions": wl.leading_positions, "d": wl.dims.d, "ffn": wl.dims.ffn,
+              "vocab": wl.dims.vocab, "heads": [wl.dims.n_q_heads, wl.dims.n_kv_heads, wl.dims.head_dim],
+              "logits_dtype": wl.logits_dtype, "parallelism": f"replicas x{args.gpus} (no collective)",
+              "l2": "weights streamed per step (>= 734 MB) exceed the 126 MB L2; no flush needed"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        steps = max(1, min(args.steps, 3))
+        warm = max(1, min(args.warmup, 1))
+        cb = run_oracle_sample(wl, steps, warm)
+        line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": UNIT, "n_gpus": args.gpus,
+                "steps": steps, "warmup": warm, "ms_per_step": cb["ms_per_bench_step"], "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
+                "cpu_baseline": {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")},
+                "e2e": {"value": cb["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line))
+        return
+
+    import torch
+    from paper_2509_23928_b200 import Drafter, hivis_profile_begin, hivis_profile_end
+    from tests.harness import to_dev, dev_weights  # device placement helpers only
+
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if world > 1:
+        wl = hi.scaled(wl, seed=wl.seed + 100 * rank)      # independent replicas, same shapes
+
+    # ---------------- set-up (untimed): weights, prompt, prefill
+    W = hi.make_weights(wl.dims, wl.seed)
+    ids, hidden, cu = hi.make_prompt(wl)
+    resid = hi.make_residuals(wl)
+    lens = np.diff(cu)
+    B, k, V = wl.batch, wl.k, wl.dims.vocab
+    dW = dev_weights(W, wl.dims.dtype)
+    del W
+    dr = Drafter(wl.dims, dW, max_batch=B, max_len=int(lens.max()) + k + 8, max_k=max(k, 8))
+    del dW
+    torch.cuda.empty_cache()
+    d_ids = torch.from_numpy(ids).cuda()
+    d_hidden = to_dev(hidden, wl.dims.dtype)
+    d_resid = to_dev(resid, wl.dims.dtype)
+    dr.prefill(d_ids, d_hidden, [int(x) for x in cu], resid0=d_resid[0])
+    out_ids = torch.empty((B, k), dtype=torch.int32, device="cuda")
+    # target logits with planted accept lengths, built from the ids of one untimed draft
+    dr.draft(B, k, d_resid, out_ids=out_ids)
+    torch.cuda.synchronize()
+    logits_np, planted = hi.make_target_logits(wl, out_ids.cpu().numpy())
+    d_logits = to_dev(logits_np, wl.logits_dtype)
+    acc = torch.empty(B, dtype=torch.int32, device="cuda")
+    nxt = torch.empty(B, dtype=torch.int32, device="cuda")
+    kvl = torch.empty(B, dtype=torch.int32, device="cuda")
+    from paper_2509_23928_b200 import hivis_verify, hivis_draft, HIVIS_BF16, HIVIS_F32
+    ldt = HIVIS_BF16 if wl.logits_dtype == "bf16" else HIVIS_F32
+    stream = torch.cuda.current_stream()
+
+    def restore():
+        for b in range(B):
+            dr.set_kv_len(b, int(lens[b]) - 1, restore_pending=True)
+
+    def one_step():
+        hivis_draft(dr.ctx, B, None, k, d_resid, d_resid.shape[0], out_ids, None, None, stream)
+        hivis_verify(dr.ctx, B, None, k, out_ids, d_logits, ldt, acc, nxt, kvl, stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---------------- timed region: K steps, CUDA events on the launching stream
+    for _ in range(max(args.warmup, 3)):
+        restore(); one_step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    n0 = dr.launch_count()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    draft_ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    for i in range(args.steps):
+        restore()
+        ev[i][0].record(stream)
+        hivis_draft(dr.ctx, B, None, k, d_resid, d_resid.shape[0], out_ids, None, None, stream)
+        draft_ev[i].record(stream)
+        hivis_verify(dr.ctx, B, None, k, out_ids, d_logits, ldt, acc, nxt, kvl, stream)
+        ev[i][1].record(stream)
+    barrier()
+    launches = dr.launch_count() - n0 - args.steps * B          # restore kernels sit outside the events
+    step_ms = np.array([a.elapsed_time(b) for a, b in ev])
+    draft_ms = np.array([ev[i][0].elapsed_time(draft_ev[i]) for i in range(args.steps)])
+    total_ms = float(step_ms.sum())
+    clocks = sampler.stop() if rank == 0 else None
+    if dist is not None:
+        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ok_planted = bool((acc.cpu().numpy() == planted).all())
+
+    # ---------------- per-kernel device time (separate pass: events around every launch)
+    restore()
+    hivis_profile_begin(dr.ctx)
+    reps = min(args.steps, 20)
+    for _ in range(reps):
+        hivis_draft(dr.ctx, B, None, k, d_resid, d_resid.shape[0], out_ids, None, None, stream)
+        restore()
+    prof = hivis_profile_end(dr.ctx)
+    kv_rows = [int(l) - 1 + k // 2 for l in lens]               # mid-chain cache length
+    step_bytes = dr.step_bytes(kv_rows)
+    es = 2 if wl.dims.dtype == "bf16" else 4
+    D = wl.dims
+    class_bytes = {"fuse_fc": 2 * D.d * D.d * es, "qkv": (D.q_dim + 2 * D.kv_dim) * D.d * es,
+                   "attention": sum(2 * (r + 1) * D.kv_dim * es for r in kv_rows), "o_proj": D.d * D.q_dim * es,
+                   "gate_up": 2 * D.ffn * D.d * es, "down": D.d * D.ffn * es, "lm_head_argmax": D.vocab * D.d * es}
+    peak, peak_kind = measured_peaks()
+    kern = {}
+    for name, (ms, n) in prof.items():
+        if n and name in class_bytes:
+            us = ms / n * 1e3
+            kern[name] = {"us": round(us, 2), "launches_per_step": n // (reps * k),
+                          "GBps": round(class_bytes[name] / (us * 1e-6) / 1e9, 1)}
+    dom = max((n for n in kern), key=lambda n: prof[n][0])
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": kern[dom]["GBps"], "peak": peak, "unit": "GB/s",
+                "frac": round(kern[dom]["GBps"] / peak, 4), "peak_kind": peak_kind, "traffic": None,
+                "algorithmic_bytes_per_launch": class_bytes[dom], "per_kernel": kern}
+
+    draft_us_per_step = float(np.median(draft_ms)) / k * 1e3
+    chain = {"us_per_draft_step_median": round(draft_us_per_step, 2),
+             "us_per_draft_step_min": round(float(draft_ms.min()) / k * 1e3, 2),
+             "verify_us_median": round(float(np.median(step_ms - draft_ms)) * 1e3, 2),
+             "algorithmic_bytes_per_draft_step": step_bytes,
+             "GBps": round(step_bytes / (draft_us_per_step * 1e-6) / 1e9, 1),
+             "frac_of_peak": round(step_bytes / (draft_us_per_step * 1e-6) / 1e9 / peak, 4),
+             "frac_of_8TBps": round(step_bytes / (draft_us_per_step * 1e-6) / 1e9 / 8000.0, 4),
+             "tokens_per_s": round(B / (draft_us_per_step * 1e-6), 1)}
+
+    # ---------------- end to end through the C ABI with HOST buffers
+    e2e = None
+    if not args.no_e2e:
+        h_resid = d_resid.cpu().pin_memory()
+        h_logits = d_logits.cpu().pin_memory()
+        h_ids = torch.empty((B, k), dtype=torch.int32).pin_memory()
+        h_res = torch.empty((3, B), dtype=torch.int32).pin_memory()
+        d_res = torch.empty((3, B), dtype=torch.int32, device="cuda")
+        d_resid2 = torch.empty_like(d_resid)
+        d_logits2 = torch.empty_like(d_logits)
+        n_e2e = max(3, min(args.steps, 20))
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            restore()
+            d_resid2.copy_(h_resid, non_blocking=True)
+            hivis_draft(dr.ctx, B, None, k, d_resid2, d_resid2.shape[0], out_ids, None, None, stream)
+            h_ids.copy_(out_ids, non_blocking=True)
+            d_logits2.copy_(h_logits, non_blocking=True)         # the target's logits arrive from the host
+            hivis_verify(dr.ctx, B, None, k, out_ids, d_logits2, ldt, d_res[0], d_res[1], d_res[2], stream)
+            h_res.copy_(d_res, non_blocking=True)
+            torch.cuda.synchronize()
+        t_e2e = time.perf_counter() - t0
+        if dist is not None:
+            t = torch.tensor([t_e2e], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            t_e2e = float(t.item())
+        e2e = {"value": world * n_e2e * k / t_e2e, "unit": UNIT,
+               "h2d_bytes_per_step": int(h_resid.numel() * h_resid.element_size() + h_logits.numel() * h_logits.element_size()),
+               "d2h_bytes_per_step": int(h_ids.numel() * 4 + h_res.numel() * 4), "steps": n_e2e,
+               "ms_per_step": t_e2e / n_e2e * 1e3}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        dr.close()
+        cb = run_oracle_sample(wl, 3, 1)
+        cpu_baseline = {k_: cb[k_] for k_ in ("value", "unit", "cores", "kind", "sample")}
+        cpu_baseline["us_per_step"] = round(cb["us_per_step"], 1)
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": world * args.steps * k / (total_ms * 1e-3), "unit": UNIT,
+                "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+                "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16 storage, f32 accumulate" if D.dtype == "bf16" else "f32",
+                "data": "synthetic", "config": config, "clocks": clocks, "e2e": e2e,
+                "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu_baseline,
+                "draft_chain": chain, "verify_matches_planted": ok_planted}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

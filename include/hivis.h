@@ -1,0 +1,198 @@
+/* hivis.h - C ABI of the HiViS drafter step on one NVIDIA B200 (sm_100a).
+ *
+ * The library runs the drafter side of HiViS speculative decoding: a single
+ * Llama-style decoder layer that never sees visual tokens.  Its input at each
+ * text position is an FC (2d -> d) fusion of the target VLM's hidden state
+ * with the embedding of the following token, plus a step-indexed
+ * bias-correction residual; its KV cache holds text positions only.
+ *
+ * Conventions shared by every call
+ *   - Every pointer is a DEVICE pointer unless its name ends in `_host`.
+ *   - Device pointers must be 16-byte aligned.
+ *   - All matrices are row-major [out, in]:  y = W x.
+ *   - The caller owns every buffer it passes.  hivis_init copies the weights
+ *     into library-owned memory (the caller may free its copies once the
+ *     stream has finished); hivis_destroy frees everything the library owns.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*, 0 = the
+ *     default stream) and return without waiting; outputs are valid once the
+ *     stream has been synchronised.  A context must always be used with work
+ *     ordered on one stream at a time, and is not thread-safe.
+ *   - Every function returns HIVIS_OK (0) or a negative error code and never
+ *     throws.  After an error nothing was launched unless the code is
+ *     HIVIS_ERR_CUDA.  hivis_last_error gives a text for the last failure.
+ *   - A sequence lives in a `slot` in [0, max_batch).  Batched calls take the
+ *     slots they work on in `seq_slots_host` (B ints, all different); NULL
+ *     means slots 0..B-1.
+ */
+#ifndef HIVIS_H
+#define HIVIS_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hivis_ctx hivis_ctx;
+
+enum {
+    HIVIS_OK = 0,
+    HIVIS_ERR_ARG = -1,      /* null / misaligned pointer, bad scalar argument            */
+    HIVIS_ERR_SHAPE = -2,    /* dimensions the kernels do not support                     */
+    HIVIS_ERR_DTYPE = -3,    /* unknown element type                                      */
+    HIVIS_ERR_STATE = -4,    /* call out of order (draft without a pending pair, ...)     */
+    HIVIS_ERR_CAPACITY = -5, /* would exceed max_batch / max_len / max_k                  */
+    HIVIS_ERR_CUDA = -6,     /* a CUDA runtime call failed                                */
+    HIVIS_ERR_TIMEOUT = -7,  /* a bounded device-side wait ran out                        */
+    HIVIS_ERR_NOMEM = -8     /* device or host allocation failed                          */
+};
+
+enum { HIVIS_F32 = 0, HIVIS_BF16 = 1 };
+
+#define HIVIS_MAX_BATCH 64   /* upper limit for hivis_config.max_batch */
+#define HIVIS_MAX_K 16       /* upper limit for hivis_config.max_k     */
+
+typedef struct {
+    uint32_t struct_size;    /* sizeof(hivis_config), checked                              */
+    int dtype;               /* HIVIS_F32 | HIVIS_BF16: weights, hidden states, residual   */
+                             /* rows and the KV cache are all stored in this type          */
+    int d;                   /* model width; multiple of 8                                 */
+    int n_q_heads, n_kv_heads;   /* n_q_heads % n_kv_heads == 0                            */
+    int head_dim;            /* 64 or 128                                                  */
+    int ffn;                 /* SwiGLU inner width; multiple of 8                          */
+    int vocab;
+    float rms_eps;
+    float rope_base;
+    int max_batch;           /* number of sequence slots, 1..HIVIS_MAX_BATCH               */
+    int max_len;             /* KV rows per slot                                           */
+    int max_k;               /* longest draft chain, 1..HIVIS_MAX_K                        */
+} hivis_config;
+
+/* The drafter's parameters (paper Sec. 3.2 and Algorithm 1).  `embed` and `lm_head` are the
+ * target model's own tables, which the drafter reuses.  `fc` is the semantic-fusion layer:
+ * columns [0,d) multiply the hidden feature (the paper's w1, stored transposed), columns
+ * [d,2d) the token embedding (w2).  `resid_proj` is the paper's w that projects a residual
+ * row r^i (rho_i = resid_proj * r_i); NULL means the rows passed to prefill/draft are used
+ * as given.  bq/bk/bv are optional QKV biases.                                              */
+typedef struct {
+    const void* embed;      /* [vocab, d]                    */
+    const void* lm_head;    /* [vocab, d]                    */
+    const void* fc;         /* [d, 2d]                       */
+    const void* norm1;      /* [d]  RMSNorm gain before QKV  */
+    const void* wq;         /* [n_q_heads*head_dim, d]       */
+    const void* wk;         /* [n_kv_heads*head_dim, d]      */
+    const void* wv;         /* [n_kv_heads*head_dim, d]      */
+    const void* bq;         /* nullable                      */
+    const void* bk;         /* nullable                      */
+    const void* bv;         /* nullable                      */
+    const void* wo;         /* [d, n_q_heads*head_dim]       */
+    const void* norm2;      /* [d]  RMSNorm gain before MLP  */
+    const void* w_gate;     /* [ffn, d]                      */
+    const void* w_up;       /* [ffn, d]                      */
+    const void* w_down;     /* [d, ffn]                      */
+    const void* resid_proj; /* [d, d], nullable              */
+} hivis_weights;
+
+/* Create a context on the current CUDA device: validates the configuration, copies (and
+ * re-lays-out) the weights, allocates the text-only KV cache [max_batch][n_kv_heads][max_len]
+ * [head_dim] x2 and all workspaces.  The only call that allocates device memory.
+ * Errors: ARG (null, misaligned, struct_size), SHAPE, DTYPE, CAPACITY, NOMEM, CUDA.          */
+int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w, void* stream);
+
+/* Waits for the device to finish and frees everything the context owns.  NULL is allowed.   */
+int hivis_destroy(hivis_ctx* ctx);
+
+/* Prefix build (Algorithm 1, lines 1-2; Eq. 1).  Appends text positions to B sequences.
+ * The batch is packed: sequence b owns entries [cu_seqlens_host[b], cu_seqlens_host[b+1]) of
+ * `ids` (int32) and of `hidden` ([total, d], ctx dtype), T_b >= 1 entries each.  Entry p is
+ * the pair (target hidden state of text token p, id of text token p+1): the causal shift of
+ * Sec. 3.2 is already applied by the caller.  For every pair but the last of each sequence
+ * the library computes fuse -> +rho_0 -> RMSNorm -> K,V projections -> RoPE(K) and stores the
+ * K/V rows (with one decoder layer nothing else of a prefix position is ever read).  The last
+ * pair of each sequence is kept as the PENDING pair that draft step 0 consumes.
+ * start_pos_host: NULL appends after the rows the slot holds now; otherwise start_pos_host[b]
+ * (0 <= start <= current length) first truncates the slot to that many rows, which lets the
+ * caller overwrite rows that came from drafting by rows built from true target features.
+ * resid0: [d] in ctx dtype = the initial residual r^0 (projected by resid_proj when the
+ * context has one); NULL = no residual.
+ * Errors: ARG, STATE, CAPACITY (rows + T_b - 1 + max... > max_len), CUDA.                    */
+int hivis_prefill(hivis_ctx* ctx, int B, const int* seq_slots_host, const int32_t* ids,
+                  const void* hidden, const int32_t* cu_seqlens_host,
+                  const int32_t* start_pos_host, const void* resid0, void* stream);
+
+/* k chained greedy draft steps for B sequences (Algorithm 1, lines 3-7; Eq. 2).  Step 0 runs
+ * the pending pair at the next cache row; step s >= 1 runs (the layer output of step s-1, the
+ * token chosen at step s-1).  Each step: fuse + residual row min(s, n_resid-1) (rows beyond
+ * the trained ones reuse the last, "Training Setup"), RMSNorm, QKV, RoPE, causal attention
+ * over the slot's cache, O projection, SwiGLU MLP, LM head, argmax (lowest index on ties).
+ * Every step appends one K/V row, so the slot grows by k rows.
+ * resid: [n_resid, d] in ctx dtype (projected by resid_proj when present); NULL = none.
+ * out_ids: int32 [B, k].
+ * forced_ids (nullable, int32 [B, k]): teacher forcing for parity tests - the token fed to
+ * step s+1 is forced_ids[b, s]; out_ids still reports each step's own argmax.
+ * out_logits (nullable, fp32 [B, k, vocab]): every step's LM-head output.
+ * Errors: ARG, STATE (a listed slot has no pending pair), CAPACITY (k > max_k or the slot
+ * would exceed max_len), CUDA.                                                                */
+int hivis_draft(hivis_ctx* ctx, int B, const int* seq_slots_host, int k, const void* resid,
+                int n_resid, int32_t* out_ids, const int32_t* forced_ids, float* out_logits,
+                void* stream);
+
+/* Batched greedy verification and KV rollback (Sec. 2.1; Algorithm 1, lines 8-9).
+ * target_logits: [B, k+1, vocab] in logits_dtype (HIVIS_F32 | HIVIS_BF16); row j is the
+ * target's prediction after the root token and j draft tokens.  Draft token j (0-based) is
+ * accepted iff it equals argmax(row j) (lowest index on ties) and all earlier ones were.
+ * out_accept[b] = n in [0, k]; out_next[b] = argmax(row n) (correction or bonus token);
+ * the slot is rolled back to (rows before the draft) + 1 + min(n, k-1) rows, also written to
+ * out_kv_len[b] (nullable).  The pending pair is consumed.  Must follow a hivis_draft of the
+ * same k on the same slots.
+ * Errors: ARG, DTYPE, STATE, CUDA.                                                            */
+int hivis_verify(hivis_ctx* ctx, int B, const int* seq_slots_host, int k,
+                 const int32_t* draft_ids, const void* target_logits, int logits_dtype,
+                 int32_t* out_accept, int32_t* out_next, int32_t* out_kv_len, void* stream);
+
+/* Forget a sequence: zero rows, no pending pair.                                              */
+int hivis_reset(hivis_ctx* ctx, int slot, void* stream);
+
+/* Synchronises `stream` and reports the slot's row count and whether a pending pair exists.  */
+int hivis_get_kv_len(hivis_ctx* ctx, int slot, int* n_rows_host, int* pending_host, void* stream);
+
+/* Set the slot's row count (0 <= n_rows <= max_len) without touching the cached data; with
+ * restore_pending != 0 the pair stored by the last prefill becomes pending again.  Lets a
+ * benchmark return to the state right after prefill between timed repetitions.               */
+int hivis_set_kv_len(hivis_ctx* ctx, int slot, int n_rows, int restore_pending, void* stream);
+
+/* Debug: copy rows [row0, row0+n) of the slot's K and V cache, widened to fp32, into
+ * out_k / out_v, each [n, n_kv_heads*head_dim].                                               */
+int hivis_read_kv(hivis_ctx* ctx, int slot, int row0, int n, float* out_k, float* out_v,
+                  void* stream);
+
+/* Debug: copy an intermediate of the LAST draft step of the last hivis_draft call, fp32,
+ * [B, width] in call order: U fused input (d), ATTN attention output (n_q_heads*head_dim),
+ * Y post-attention residual (d), ACT SwiGLU product (ffn), G layer output (d).               */
+enum { HIVIS_TAP_U = 0, HIVIS_TAP_ATTN = 1, HIVIS_TAP_Y = 2, HIVIS_TAP_ACT = 3, HIVIS_TAP_G = 4 };
+int hivis_debug_tap(hivis_ctx* ctx, int which, float* out, void* stream);
+
+/* Per-kernel timing of hivis_draft.  Between hivis_profile_begin and hivis_profile_end every
+ * kernel the draft chain launches is bracketed by CUDA events on its stream (this slows the chain
+ * slightly, so time whole chains without it).  hivis_profile_end waits for the last event and adds
+ * up, per kernel class, the device time in ms and the number of launches; both arrays are host
+ * arrays of HIVIS_PROFILE_CLASSES entries, indexed: 0 fuse FC, 1 QKV, 2 attention, 3 O projection,
+ * 4 gate/up, 5 down, 6 LM head + argmax, 7 set-up and finish kernels.                          */
+#define HIVIS_PROFILE_CLASSES 8
+int hivis_profile_begin(hivis_ctx* ctx);
+int hivis_profile_end(hivis_ctx* ctx, float* ms_host, int64_t* launches_host);
+
+/* Bytes of weights and KV that one draft step of the given batch must read at least once
+ * (the roofline's numerator): weights once per step regardless of B, plus K and V rows
+ * [0, rows_b] of every listed slot.  kv_rows_host[b] = rows the slot holds at that step.      */
+int64_t hivis_step_bytes(const hivis_ctx* ctx, int B, const int* kv_rows_host);
+
+/* Number of kernel launches the library has enqueued since the context was created.          */
+int64_t hivis_launch_count(const hivis_ctx* ctx);
+
+const char* hivis_last_error(const hivis_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HIVIS_H */

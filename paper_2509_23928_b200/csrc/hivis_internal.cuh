@@ -1,0 +1,192 @@
+// Internal declarations shared by the kernel files and the host layer of libhivis.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/hivis.h"
+
+typedef __nv_bfloat16 bf16;
+typedef unsigned long long u64;
+
+// ---------------------------------------------------------------------------------------------
+// Skinny linear layer  out[b][n] = sum_k W[n][k] * x[b][k]  with a fused input stage (PRO_*)
+// and a fused output stage (EPI_*).  Two kernel families share these arguments:
+//   gemv_alu : fp32 FMAs, one batch row per CTA column (B == 1, or fp32 weights)
+//   gemm_mma : bf16 tensor-core tiles, up to 16 batch rows per pass
+// ---------------------------------------------------------------------------------------------
+enum { PRO_PLAIN = 0, PRO_NORM = 1, PRO_FUSE = 2 };
+enum { EPI_FUSE = 0, EPI_QKV = 1, EPI_OPROJ = 2, EPI_GATEUP = 3, EPI_DOWN = 4, EPI_LM = 5 };
+
+struct LinArgs {
+    const void* W;        // [N][K] in the context dtype
+    int N, K, B;
+    int ldb;              // row stride (elements) of the ssq buffers = batch capacity
+    // ---- input stage
+    const float* xin;     // PRO_PLAIN / PRO_NORM (alu): [B][K] fp32
+    const bf16* xin_h;    // mma: [B][K] bf16 (already multiplied by the norm gain where one applies)
+    const void* gamma;    // PRO_NORM (alu): [K] gain, context dtype
+    float eps;
+    const float* feat;    // PRO_FUSE (alu): [B][d] fp32 hidden feature
+    const void* feat_h;   // PRO_FUSE (mma): [B][d] bf16 hidden feature
+    const void* embed;    // PRO_FUSE: [vocab][d], context dtype
+    const int* ids;       // PRO_FUSE: token of row b = ids[b * id_stride]; if null, decoded from keys
+    int id_stride;
+    const u64* keys;      // PRO_FUSE: packed argmax keys, row b at keys[b * key_stride]
+    int key_stride;
+    int d;
+    // ---- scale recovered from per-tile partial sums of squares (mma EPI_QKV / EPI_GATEUP):
+    //      s[b] = rsqrt( sum_t ssq_in[t*ldb + b] / K + eps )
+    const float* ssq_in;
+    int ssq_tiles;
+    // ---- output stage
+    const void* bias;     // EPI_QKV: [N] context dtype, nullable
+    const float* rho;     // EPI_FUSE: [N] fp32 residual row, nullable
+    const float* addend;  // EPI_OPROJ (u), EPI_DOWN (y): [B][N] fp32
+    float* out;           // fp32 result [B][N] (EPI_GATEUP: [B][N/2]); nullable
+    bf16* out_h;          // bf16 copy [B][N] (EPI_GATEUP: [B][N/2]); nullable
+    const void* gamma_out;// EPI_FUSE / EPI_OPROJ: out_h = bf16(gamma_out[n] * value), context dtype
+    float* ssq_out;       // EPI_FUSE / EPI_OPROJ (mma): [tiles][ldb] partial sums of squares
+    u64* keys_out;        // EPI_LM: row b at keys_out[b * keys_out_stride]
+    int keys_out_stride;
+    float* logits_out;    // EPI_LM: nullable, row b at logits_out[b * logits_ld]
+    long long logits_ld;
+};
+
+// Rows of W covered by one CTA of the tensor-core kernel.
+#define HIVIS_MMA_TILE_ROWS 32
+
+cudaError_t launch_gemv_alu(int dtype, int pro, int epi, const LinArgs& a, cudaStream_t st);
+cudaError_t launch_gemm_mma(int pro, int epi, const LinArgs& a, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------
+// Decode attention over the text-only cache (one new position per sequence).
+// ---------------------------------------------------------------------------------------------
+struct AttnArgs {
+    const float* qkv;     // [B][ld]: q | k | v of the new position, before RoPE
+    int ld;
+    void* Kc;             // [slot][Hkv][max_len][dh], context dtype, K stored after RoPE
+    void* Vc;
+    const int* slots;     // [B]
+    const int* pos0;      // [B] cache row of draft step 0
+    int step;             // this step's row = pos0[b] + step
+    const double* inv_freq;   // [dh/2]  base^(-2i/dh)
+    int Hq, Hkv, dh, max_len, B;
+    float scale;          // 1/sqrt(dh)
+    int chunk;            // cache rows per split
+    int nsplit;           // grid.x
+    float* part_acc;      // [B][Hq][nsplit][dh]
+    float* part_ml;       // [B][Hq][nsplit][2]
+    int* counters;        // [B][Hq] arrival counters, zero between launches
+    float* attn;          // [B][Hq*dh] fp32
+    bf16* attn_h;         // [B][Hq*dh] bf16 copy
+};
+cudaError_t launch_attention(int dtype, const AttnArgs& a, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------
+// Small kernels: state set-up, prefill bookkeeping, verification, layout changes, taps.
+// ---------------------------------------------------------------------------------------------
+struct SlotList {
+    int n;
+    int slot[HIVIS_MAX_BATCH];
+};
+struct CuSeqlens {
+    int v[HIVIS_MAX_BATCH + 1];
+};
+
+// draft set-up: slots -> device, pos0 = kv_len[slot], feat = pending feature, ids = pending id;
+// clears the argmax keys [B][k]; advances kv_len by k.
+cudaError_t launch_draft_setup(const SlotList& sl, int k, int d, int* d_slots, int* d_pos0,
+                               int* kv_len, const float* pend_feat, const int* pend_id, float* feat,
+                               bf16* feat_h, int* cur_id, u64* keys, int key_stride, cudaStream_t st);
+// decode keys [B][k] into out_ids [B][k]
+cudaError_t launch_draft_finish(int B, int k, const u64* keys, int key_stride, int32_t* out_ids,
+                                cudaStream_t st);
+
+// residual rows (context dtype) -> fp32 rho [R][d] (no projection)
+cudaError_t launch_convert_rows(int dtype, const void* src, float* dst, long long n, cudaStream_t st);
+cudaError_t launch_f32_to_bf16(const float* src, bf16* dst, long long n, cudaStream_t st);
+cudaError_t launch_bf16_to_f32(const bf16* src, float* dst, long long n, cudaStream_t st);
+
+// prefill bookkeeping: for every packed entry j: slot_of[j], row_of[j] (-1 for the pending pair);
+// stores the pending pair; updates kv_len.
+cudaError_t launch_prefill_setup(int dtype, const SlotList& sl, const CuSeqlens& cu,
+                                 const SlotList& start /* -1 = append */, int d, const int32_t* ids,
+                                 const void* hidden, int* kv_len, float* pend_feat, int* pend_id,
+                                 int* slot_of, int* row_of, cudaStream_t st);
+// RoPE(K) and store K,V rows of a chunk of packed entries
+cudaError_t launch_kv_append(int dtype, const float* kv /*[P][2*kvw]*/, int P, const int* slot_of,
+                             const int* row_of, const double* inv_freq, int Hkv, int dh, int max_len,
+                             void* Kc, void* Vc, cudaStream_t st);
+
+// verification: row argmax over [B][k+1][V], then accept length / next token / rollback
+cudaError_t launch_verify(int logits_dtype, const SlotList& sl, int k, int V, const int32_t* draft_ids,
+                          const void* logits, u64* keys, int* kv_len, int32_t* out_accept,
+                          int32_t* out_next, int32_t* out_kv_len, cudaStream_t st, int* n_launches);
+
+cudaError_t launch_set_int(int* p, int v, cudaStream_t st);
+
+// weight re-layout at init
+cudaError_t launch_copy_rows(const void* src, void* dst, long long rows, long long row_bytes,
+                             long long dst_row0, long long dst_row_step, cudaStream_t st);
+
+cudaError_t launch_read_kv(int dtype, const void* Kc, const void* Vc, int slot, int row0, int n,
+                           int Hkv, int dh, int max_len, float* out_k, float* out_v, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------
+// device helpers
+// ---------------------------------------------------------------------------------------------
+#ifdef __CUDACC__
+// Order-preserving map of a float to 32 bits (NaN -> 0 so that it never wins), packed with the
+// index so that a 64-bit integer max picks the largest value and, among equals, the lowest index.
+__device__ __forceinline__ u64 pack_key(float v, int idx) {
+    unsigned int u = __float_as_uint(v);
+    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    if (v != v) u = 0u;
+    return ((u64)u << 32) | (u64)(0xFFFFFFFFu - (unsigned int)idx);
+}
+__device__ __forceinline__ int key_index(u64 key) {
+    return (int)(0xFFFFFFFFu - (unsigned int)(key & 0xFFFFFFFFull));
+}
+__device__ __forceinline__ float bf16_lo(unsigned int w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(unsigned int w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+template <typename WT>
+__device__ __forceinline__ float load_as_float(const void* p, long long i);
+template <>
+__device__ __forceinline__ float load_as_float<float>(const void* p, long long i) {
+    return ((const float*)p)[i];
+}
+template <>
+__device__ __forceinline__ float load_as_float<bf16>(const void* p, long long i) {
+    return __bfloat162float(((const bf16*)p)[i]);
+}
+template <typename WT>
+__device__ __forceinline__ void store_from_float(void* p, long long i, float v);
+template <>
+__device__ __forceinline__ void store_from_float<float>(void* p, long long i, float v) {
+    ((float*)p)[i] = v;
+}
+template <>
+__device__ __forceinline__ void store_from_float<bf16>(void* p, long long i, float v) {
+    ((bf16*)p)[i] = __float2bfloat16_rn(v);
+}
+
+// 16-byte streaming load of weights: read-only path, do not keep in L1.
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+// 16-byte load of an activation written by an earlier kernel: L2 only.
+__device__ __forceinline__ uint4 ld_act(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+#endif

@@ -1,0 +1,275 @@
+"""GPU parity: the CUDA library against the CPU oracle on the same seeded inputs, through the C ABI."""
+import numpy as np
+import pytest
+
+import hivis_inputs as hi
+from tests.harness import Case, check_draft_parity, check_kv_parity, check_verify_parity, to_dev, row_rel_err
+
+pytestmark = pytest.mark.gpu
+
+SMALL = ["c1_tiny_f32_b1", "mini_mha_b1", "mini_mha_b5_ragged", "mini_gqa_b16_ragged", "mini_gqa_b3",
+         "tiny_f32_b4_ragged"]
+
+
+@pytest.mark.parametrize("name", SMALL)
+def test_draft_kv_verify_parity_small(name):
+    case = Case(hi.workload(name))
+    try:
+        res = check_draft_parity(case)
+        check_kv_parity(case, res["ref"])              # cache after the teacher-forced run = oracle's run
+        check_verify_parity(case, res["ids_o"])
+    finally:
+        case.close()
+
+
+def test_c1_ids_exact_and_tight_logits():
+    case = Case(hi.workload("c1_tiny_f32_b1"))
+    try:
+        res = check_draft_parity(case, rtol=1e-4)
+        assert res["excused"] == 0
+        np.testing.assert_array_equal(res["ids_g"], res["ids_o"])
+    finally:
+        case.close()
+
+
+def test_intermediate_taps_match_oracle():
+    wl = hi.workload("mini_mha_b5_ragged")
+    case = Case(wl)
+    try:
+        case.gpu_prefill()
+        case.gpu_draft(1)
+        rho = case.oracle.fold_residuals(case.resid)
+        for b in range(wl.batch):
+            lo, hi_ = int(case.cu[b]), int(case.cu[b + 1])
+            T = hi_ - lo
+            Kc, Vc = case.oracle.new_cache(T + 1)
+            case.oracle.prefill(case.ids[lo:hi_], case.hidden[lo:hi_], rho[0], Kc, Vc)
+            _, taps = case.oracle.position(case.hidden[hi_ - 1], int(case.ids[hi_ - 1]), rho[0], T - 1, Kc, Vc, taps=True)
+            for name in ("u", "attn", "y", "act", "g"):
+                got = case.drafter.tap(name, wl.batch)[b].cpu().numpy()
+                e = np.abs(got - taps[name]).max() / np.abs(taps[name]).max()
+                assert e < 2e-2, f"tap {name} seq {b}: rel err {e}"
+    finally:
+        case.close()
+
+
+@pytest.mark.parametrize("T,k", [(1, 1), (1, 5), (2, 3), (129, 2), (128, 4), (257, 1)])
+def test_edge_lengths(T, k):
+    wl = hi.scaled(hi.workload("mini_mha_b1"), text_len=T, k=k, seed=3000 + T + k)
+    case = Case(wl)
+    try:
+        res = check_draft_parity(case)
+        check_kv_parity(case, res["ref"])
+        check_verify_parity(case, res["ids_o"])
+    finally:
+        case.close()
+
+
+def test_qkv_bias_and_residual_projection():
+    wl = hi.workload("mini_gqa_b3")
+    rng = np.random.default_rng(5)
+    D = wl.dims
+    extra = {"bq": hi.round_to_bf16(rng.standard_normal(D.q_dim).astype(np.float32) * 0.5),
+             "bk": hi.round_to_bf16(rng.standard_normal(D.kv_dim).astype(np.float32) * 0.5),
+             "bv": hi.round_to_bf16(rng.standard_normal(D.kv_dim).astype(np.float32) * 0.5)}
+    case = Case(wl, extra_weights=extra)
+    try:
+        res = check_draft_parity(case)
+        check_kv_parity(case, res["ref"])
+    finally:
+        case.close()
+
+
+def test_residual_projection_matrix():
+    import torch
+    from paper_2509_23928_b200 import Drafter
+    from tests.harness import dev_weights
+    import oracle
+    wl = hi.workload("mini_mha_b1")
+    D = wl.dims
+    W = hi.make_weights(D, wl.seed)
+    rp = hi.round_to_bf16(np.random.default_rng(6).standard_normal((D.d, D.d)).astype(np.float32) * 0.05)
+    ids, hidden, cu = hi.make_prompt(wl)
+    resid = hi.make_residuals(wl)
+    o = oracle.Oracle(D, W)
+    ref = o.run_batch(ids, hidden, cu, wl.k, resid, resid_proj=rp)[0]
+    dW = dev_weights(W, "bf16")
+    dW["resid_proj"] = to_dev(rp, "bf16")
+    dr = Drafter(D, dW, 1, 64, 8)
+    try:
+        d_resid = to_dev(resid, "bf16")
+        dr.prefill(torch.from_numpy(ids).cuda(), to_dev(hidden, "bf16"), [int(x) for x in cu], resid0=d_resid[0])
+        f = torch.from_numpy(ref["ids"][None].astype(np.int32)).cuda()
+        _, logits = dr.draft(1, wl.k, d_resid, forced_ids=f, want_logits=True)
+        torch.cuda.synchronize()
+        assert row_rel_err(logits[0].cpu().numpy(), ref["logits"]).max() < 2e-2
+    finally:
+        dr.close()
+
+
+def test_no_residual_equals_zero_residual():
+    import torch
+    wl = hi.workload("mini_mha_b1")
+    case = Case(wl)
+    try:
+        case.drafter.prefill(case.d_ids, case.d_hidden, [int(x) for x in case.cu], resid0=None)
+        ids_a, la = case.drafter.draft(1, 3, None, want_logits=True)
+        case.gpu_restore()
+        z = torch.zeros_like(case.d_resid)
+        case.drafter.prefill(case.d_ids, case.d_hidden, [int(x) for x in case.cu], start_pos=[0], resid0=z[0])
+        ids_b, lb = case.drafter.draft(1, 3, z, want_logits=True)
+        torch.cuda.synchronize()
+        assert torch.equal(ids_a, ids_b) and torch.equal(la, lb)
+    finally:
+        case.close()
+
+
+def test_run_to_run_determinism():
+    wl = hi.workload("mini_gqa_b16_ragged")
+    case = Case(wl)
+    try:
+        case.gpu_prefill()
+        ids_a, la = case.gpu_draft()
+        case.gpu_restore()
+        ids_b, lb = case.gpu_draft()
+        np.testing.assert_array_equal(ids_a, ids_b)
+        np.testing.assert_array_equal(la, lb)
+    finally:
+        case.close()
+
+
+def test_slots_subset_and_order():
+    """Sequences may sit in any slots, in any order, and calls may address a subset."""
+    import torch
+    wl = hi.workload("mini_mha_b5_ragged")
+    case = Case(wl)
+    try:
+        ref = case.oracle_run()
+        perm = [3, 0, 4, 1, 2]
+        # prefill sequence b into slot perm[b]
+        case.drafter.prefill(case.d_ids, case.d_hidden, [int(x) for x in case.cu], slots=perm, resid0=case.d_resid[0])
+        sub = [1, 3]                                  # draft only sequences 1 and 3, listed in reverse
+        slots = [perm[3], perm[1]]
+        ids = case.drafter.draft(2, wl.k, case.d_resid, slots=slots)
+        torch.cuda.synchronize()
+        ids = ids.cpu().numpy()
+        for row, b in enumerate([3, 1]):
+            first_bad = next((s for s in range(wl.k) if ids[row, s] != ref[b]["ids"][s]), None)
+            assert first_bad is None or ref[b]["gaps"][first_bad] < 1e-2
+        assert case.drafter.kv_len(perm[3])[0] == case.lens[3] - 1 + wl.k
+        assert case.drafter.kv_len(perm[0])[0] == case.lens[0] - 1      # untouched
+    finally:
+        case.close()
+
+
+def test_multi_round_loop_with_refresh_matches_oracle():
+    """draft -> verify -> prefill(start_pos) refresh -> draft, compared with the oracle doing the same."""
+    import torch
+    wl = hi.workload("mini_mha_b1")
+    case = Case(wl, max_len=128)
+    try:
+        o, D = case.oracle, wl.dims
+        k = 4
+        rho = o.fold_residuals(case.resid)
+        T = int(case.lens[0])
+        Kc, Vc = o.new_cache(128)
+        o.prefill(case.ids, case.hidden, rho[0], Kc, Vc)
+        case.gpu_prefill()
+        pend_h, pend_id = case.hidden[-1], int(case.ids[-1])
+        rng = np.random.default_rng(77)
+        for rnd in range(3):
+            ref = o.draft(T - 1, pend_id, pend_h, k, rho, Kc, Vc)
+            f = torch.from_numpy(ref["ids"][None].astype(np.int32)).cuda()
+            ids_g, logits_g = case.drafter.draft(1, k, case.d_resid, forced_ids=f, want_logits=True)
+            torch.cuda.synchronize()
+            assert row_rel_err(logits_g[0].cpu().numpy(), ref["logits"]).max() < 2e-2, f"round {rnd}"
+            planted = np.array([[2, 0, 4][rnd]])
+            logits, _ = hi.make_target_logits(hi.scaled(wl, k=k, seed=wl.seed + rnd), ref["ids"][None], planted)
+            acc, nxt, kv = case.drafter.verify(f, to_dev(logits, wl.logits_dtype))
+            torch.cuda.synchronize()
+            n, nx, kvl = o.verify(ref["ids"], logits[0], T)
+            assert (int(acc[0]), int(nxt[0]), int(kv[0])) == (n, nx, kvl)
+            # the target now supplies hidden states for the n+1 new tokens; refresh rows T.. with them
+            new_ids = np.array(list(ref["ids"][:n]) + [nx], np.int32)
+            new_hidden = hi.round_to_bf16(rng.standard_normal((n + 1, D.d)).astype(np.float32))
+            o.prefill(new_ids, new_hidden, rho[0], Kc, Vc, start_pos=T)
+            case.drafter.prefill(torch.from_numpy(new_ids).cuda(), to_dev(new_hidden, "bf16"), [0, n + 1],
+                                 start_pos=[T], resid0=case.d_resid[0])
+            T += n + 1
+            pend_h, pend_id = new_hidden[-1], int(new_ids[-1])
+            assert case.drafter.kv_len(0) == (T - 1, True)
+        k_g, v_g = case.drafter.read_kv(0, 0, T - 1)
+        torch.cuda.synchronize()
+        assert np.abs(k_g.cpu().numpy() - Kc[:T - 1]).max() / np.abs(Kc[:T - 1]).max() < 1e-2
+        assert np.abs(v_g.cpu().numpy() - Vc[:T - 1]).max() / np.abs(Vc[:T - 1]).max() < 1e-2
+    finally:
+        case.close()
+
+
+def test_verify_ties_bf16_and_unaligned_vocab():
+    """bf16 logits make exact ties common: the lowest index must win on both sides."""
+    import torch
+    wl = hi.scaled(hi.workload("mini_gqa_b3"), k=3)         # vocab 5031: rows are not 16-byte aligned
+    case = Case(wl)
+    try:
+        case.gpu_prefill()
+        ids_g, _ = case.gpu_draft(3, want_logits=False)
+        V = wl.dims.vocab
+        rng = np.random.default_rng(8)
+        logits = hi.round_to_bf16(rng.integers(-3, 4, size=(3, 4, V)).astype(np.float32))   # massive ties
+        d_logits = to_dev(logits, "bf16")
+        d_ids = torch.from_numpy(ids_g).cuda()
+        acc, nxt, kv = case.drafter.verify(d_ids, d_logits)
+        torch.cuda.synchronize()
+        for b in range(3):
+            n, nx, kvl = case.oracle.verify(ids_g[b], logits[b], int(case.lens[b]))
+            assert (int(acc[b]), int(nxt[b]), int(kv[b])) == (n, nx, kvl)
+            assert nx == int(np.argmax(logits[b, n]))
+    finally:
+        case.close()
+
+
+def test_host_side_errors_do_not_launch():
+    import torch
+    from paper_2509_23928_b200 import HivisError
+    wl = hi.workload("c1_tiny_f32_b1")
+    case = Case(wl, max_len=40, max_k=4)
+    try:
+        dr = case.drafter
+        n0 = dr.launch_count()
+        out = torch.empty((1, 4), dtype=torch.int32, device="cuda")
+        with pytest.raises(HivisError) as e:                     # draft before prefill
+            dr.draft(1, 4, case.d_resid, out_ids=out)
+        assert e.value.code == -4
+        with pytest.raises(HivisError) as e:                     # k beyond max_k
+            dr.draft(1, 5, case.d_resid)
+        assert e.value.code == -5
+        with pytest.raises(HivisError) as e:                     # slot out of range
+            dr.draft(1, 2, case.d_resid, slots=[3])
+        assert e.value.code == -1
+        with pytest.raises(HivisError) as e:                     # duplicate slot / too many sequences
+            dr.prefill(case.d_ids, case.d_hidden, [0, 16, 32], resid0=None)
+        assert e.value.code == -5
+        with pytest.raises(HivisError) as e:                     # misaligned pointer
+            dr.prefill(case.d_ids[1:], case.d_hidden, [0, 31])
+        assert e.value.code == -1
+        assert dr.launch_count() == n0
+        case.gpu_prefill()                                       # 31 rows + pending
+        with pytest.raises(HivisError) as e:                     # would overflow max_len = 40 ... 31 + 4 fits; shrink
+            dr.set_kv_len(0, 41)
+        assert e.value.code == -5
+        dr.set_kv_len(0, 38, restore_pending=True)
+        with pytest.raises(HivisError) as e:
+            dr.draft(1, 4, case.d_resid)                         # 38 + 4 > 40
+        assert e.value.code == -5
+        dr.set_kv_len(0, 31, restore_pending=True)
+        ids = dr.draft(1, 4, case.d_resid)
+        logits = torch.zeros((1, 4, wl.dims.vocab), device="cuda")
+        with pytest.raises(HivisError) as e:                     # verify with another k
+            dr.verify(ids[:, :3].contiguous(), logits)
+        assert e.value.code == -4
+        with pytest.raises(HivisError) as e:                     # second draft without a pending pair
+            dr.draft(1, 4, case.d_resid)
+        assert e.value.code == -4
+    finally:
+        case.close()
