@@ -280,8 +280,9 @@ def main():
         h_resid = d_resid.cpu().pin_memory()
         h_logits = d_logits.cpu().pin_memory()
         h_ids = torch.empty((B, k), dtype=torch.int32).pin_memory()
-        h_res = torch.empty((3, B), dtype=torch.int32).pin_memory()
-        d_res = torch.empty((3, B), dtype=torch.int32, device="cuda")
+        Bp = (B + 3) // 4 * 4                                    # rows stay 16-byte aligned
+        h_res = torch.empty((3, Bp), dtype=torch.int32).pin_memory()
+        d_res = torch.empty((3, Bp), dtype=torch.int32, device="cuda")
         d_resid2 = torch.empty_like(d_resid)
         d_logits2 = torch.empty_like(d_logits)
         n_e2e = max(3, min(args.steps, 20))
@@ -303,7 +304,7 @@ def main():
             t_e2e = float(t.item())
         e2e = {"value": world * n_e2e * k / t_e2e, "unit": UNIT,
                "h2d_bytes_per_step": int(h_resid.numel() * h_resid.element_size() + h_logits.numel() * h_logits.element_size()),
-               "d2h_bytes_per_step": int(h_ids.numel() * 4 + h_res.numel() * 4), "steps": n_e2e,
+               "d2h_bytes_per_step": int(h_ids.numel() * 4 + 3 * B * 4), "steps": n_e2e,
                "ms_per_step": t_e2e / n_e2e * 1e3}
 
     cpu_baseline = None
