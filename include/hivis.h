@@ -172,13 +172,27 @@ int hivis_read_kv(hivis_ctx* ctx, int slot, int row0, int n, float* out_k, float
 enum { HIVIS_TAP_U = 0, HIVIS_TAP_ATTN = 1, HIVIS_TAP_Y = 2, HIVIS_TAP_ACT = 3, HIVIS_TAP_G = 4 };
 int hivis_debug_tap(hivis_ctx* ctx, int which, float* out, void* stream);
 
+/* Options.  HIVIS_OPT_CHAIN_KERNEL (default 1): a draft of ONE sequence runs all k steps in a
+ * single persistent cooperative kernel (one CTA per SM, grid barriers between the phases of a step,
+ * weights prefetched across them); 0 runs the same steps as separate kernel launches, which is what
+ * batches of two or more sequences always use.  Both give the same results up to fp32 summation
+ * order.                                                                                        */
+enum { HIVIS_OPT_CHAIN_KERNEL = 0 };
+int hivis_set_option(hivis_ctx* ctx, int option, int value);
+
+/* Synchronises `stream` and reports whether any kernel since the last call gave up on a bounded
+ * device-side wait (HIVIS_ERR_TIMEOUT; the outputs of that call are invalid, the context stays
+ * usable).  Otherwise HIVIS_OK.                                                                 */
+int hivis_status(hivis_ctx* ctx, void* stream);
+
 /* Per-kernel timing of hivis_draft.  Between hivis_profile_begin and hivis_profile_end every
  * kernel the draft chain launches is bracketed by CUDA events on its stream (this slows the chain
  * slightly, so time whole chains without it).  hivis_profile_end waits for the last event and adds
  * up, per kernel class, the device time in ms and the number of launches; both arrays are host
  * arrays of HIVIS_PROFILE_CLASSES entries, indexed: 0 fuse FC, 1 QKV, 2 attention, 3 O projection,
- * 4 gate/up, 5 down, 6 LM head + argmax, 7 set-up and finish kernels.                          */
-#define HIVIS_PROFILE_CLASSES 8
+ * 4 gate/up, 5 down, 6 LM head + argmax, 7 set-up and finish kernels, 8 the persistent chain
+ * kernel (all k steps of one sequence in one launch).                                          */
+#define HIVIS_PROFILE_CLASSES 9
 int hivis_profile_begin(hivis_ctx* ctx);
 int hivis_profile_end(hivis_ctx* ctx, float* ms_host, int64_t* launches_host);
 

@@ -16,8 +16,11 @@ ERRORS = {0: "OK", -1: "ARG", -2: "SHAPE", -3: "DTYPE", -4: "STATE", -5: "CAPACI
 
 EXPORTS = ("hivis_init", "hivis_destroy", "hivis_prefill", "hivis_draft", "hivis_verify", "hivis_reset",
            "hivis_get_kv_len", "hivis_set_kv_len", "hivis_read_kv", "hivis_debug_tap", "hivis_step_bytes",
-           "hivis_launch_count", "hivis_last_error", "hivis_profile_begin", "hivis_profile_end")
-PROFILE_CLASSES = ("fuse_fc", "qkv", "attention", "o_proj", "gate_up", "down", "lm_head_argmax", "setup_finish")
+           "hivis_launch_count", "hivis_last_error", "hivis_profile_begin", "hivis_profile_end", "hivis_set_option",
+           "hivis_status")
+HIVIS_OPT_CHAIN_KERNEL = 0
+PROFILE_CLASSES = ("fuse_fc", "qkv", "attention", "o_proj", "gate_up", "down", "lm_head_argmax", "setup_finish",
+                   "draft_chain")
 
 
 class HivisError(RuntimeError):
@@ -63,6 +66,8 @@ def _load() -> C.CDLL:
     L.hivis_step_bytes.restype = C.c_int64
     L.hivis_launch_count.argtypes = [vp]
     L.hivis_launch_count.restype = C.c_int64
+    L.hivis_set_option.argtypes = [vp, i32, i32]
+    L.hivis_status.argtypes = [vp, vp]
     L.hivis_profile_begin.argtypes = [vp]
     L.hivis_profile_end.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int64)]
     L.hivis_last_error.argtypes = [vp]
@@ -162,6 +167,15 @@ def hivis_step_bytes(ctx, kv_rows: Sequence[int]) -> int:
     return int(lib.hivis_step_bytes(ctx, len(kv_rows), _ints(kv_rows)))
 
 
+def hivis_set_option(ctx, option: int, value: int) -> None:
+    _check(lib.hivis_set_option(ctx, int(option), int(value)), ctx)
+
+
+def hivis_status(ctx, stream=None) -> None:
+    """Synchronise and raise HivisError(TIMEOUT) if a kernel gave up on a bounded wait."""
+    _check(lib.hivis_status(ctx, _stream(stream)), ctx)
+
+
 def hivis_profile_begin(ctx) -> None:
     _check(lib.hivis_profile_begin(ctx), ctx)
 
@@ -256,6 +270,12 @@ class Drafter:
         out = t.empty((B, width), dtype=t.float32, device=self.dev)
         hivis_debug_tap(self.ctx, TAPS[name], out)
         return out
+
+    def set_chain_kernel(self, on: bool):
+        hivis_set_option(self.ctx, HIVIS_OPT_CHAIN_KERNEL, 1 if on else 0)
+
+    def status(self):
+        hivis_status(self.ctx)
 
     def step_bytes(self, kv_rows):
         return hivis_step_bytes(self.ctx, kv_rows)

@@ -33,6 +33,13 @@ struct hivis_ctx {
     float *part_acc, *part_ml;
     int* counters;
     int chunk, nsplit_cap;
+    // persistent chain kernel
+    int num_sms;
+    bool chain_ok;                // cooperative launch available and the kernel fits
+    bool opt_chain;               // option HIVIS_OPT_CHAIN_KERNEL
+    u64* bar_counter;
+    u64 bar_count_host;           // value of *bar_counter once everything enqueued has run
+    int* error_flag;
     int *slot_of, *row_of;
     long long map_cap;
     // host mirrors
@@ -53,7 +60,8 @@ struct hivis_ctx {
     size_t prof_n;
 };
 
-enum { CLS_FUSE = 0, CLS_QKV, CLS_ATTN, CLS_OPROJ, CLS_GATEUP, CLS_DOWN, CLS_LM, CLS_OTHER, CLS_COUNT };
+enum { CLS_FUSE = 0, CLS_QKV, CLS_ATTN, CLS_OPROJ, CLS_GATEUP, CLS_DOWN, CLS_LM, CLS_OTHER, CLS_CHAIN, CLS_COUNT };
+static_assert(CLS_COUNT == HIVIS_PROFILE_CLASSES, "profile classes");
 
 static void prof_mark(hivis_ctx* c, int cls, cudaStream_t st, bool begin) {
     if (!c->prof_on) return;
@@ -102,6 +110,10 @@ static char g_init_err[256] = "";
         (c)->launches += 1;                 \
         prof_mark(c, cls, st, false);       \
     } while (0)
+
+extern "C" {
+static void fill_chain_args(hivis_ctx* c, ChainArgs* a);
+}
 
 static bool misaligned(const void* p) { return (((uintptr_t)p) & 15u) != 0; }
 
@@ -218,7 +230,21 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
     const size_t es = c->esize;
     const long long d = cfg->d, F = cfg->ffn, V = cfg->vocab, R = c->rows_cap, MB = cfg->max_batch;
     c->chunk = 128;
-    c->nsplit_cap = (cfg->max_len + c->chunk - 1) / c->chunk;
+    c->nsplit_cap = (cfg->max_len + 31) / 32;
+    if (c->nsplit_cap > 64) c->nsplit_cap = 64;
+    c->opt_chain = true;
+    c->chain_ok = false;
+    c->bar_count_host = 0;
+    {
+        int coop = 0;
+        c->num_sms = 0;
+        if (cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess ||
+            cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device) != cudaSuccess) {
+            cudaGetLastError();
+            coop = 0;
+        }
+        c->chain_ok = coop != 0 && c->num_sms > 0;
+    }
     c->key_stride = cfg->max_k + 1;
     c->map_cap = MB * (long long)cfg->max_len;
     const long long tiles1 = (d + HIVIS_MMA_TILE_ROWS - 1) / HIVIS_MMA_TILE_ROWS;
@@ -243,7 +269,8 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
          dalloc(c, &c->ssq2, tiles1 * R) && dalloc(c, &c->keys, R * c->key_stride) &&
          dalloc(c, &c->part_acc, R * cfg->n_q_heads * (long long)c->nsplit_cap * cfg->head_dim) &&
          dalloc(c, &c->part_ml, R * cfg->n_q_heads * (long long)c->nsplit_cap * 2) &&
-         dalloc(c, &c->counters, R * cfg->n_q_heads) && dalloc(c, &c->slot_of, c->map_cap) &&
+         dalloc(c, &c->counters, R * cfg->n_q_heads) && dalloc(c, &c->bar_counter, 1) &&
+         dalloc(c, &c->error_flag, 1) && dalloc(c, &c->slot_of, c->map_cap) &&
          dalloc(c, &c->row_of, c->map_cap);
     if (!ok) {
         free_all(c);
@@ -283,6 +310,8 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
         CK(c, cudaMemsetAsync(c->kv_len, 0, MB * sizeof(int), st));
         CK(c, cudaMemsetAsync(c->pend_id, 0, MB * sizeof(int), st));
         CK(c, cudaMemsetAsync(c->counters, 0, R * cfg->n_q_heads * sizeof(int), st));
+        CK(c, cudaMemsetAsync(c->bar_counter, 0, sizeof(u64), st));
+        CK(c, cudaMemsetAsync(c->error_flag, 0, sizeof(int), st));
         CK(c, cudaMemsetAsync(c->Kc, 0, MB * c->kvw * (long long)cfg->max_len * es, st));
         CK(c, cudaMemsetAsync(c->Vc, 0, MB * c->kvw * (long long)cfg->max_len * es, st));
         return HIVIS_OK;
@@ -293,6 +322,11 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
         free_all(c);
         delete c;
         return rc;
+    }
+    if (c->chain_ok) {
+        ChainArgs ca;
+        fill_chain_args(c, &ca);
+        c->chain_ok = chain_smem_bytes(ca, c->dtype, c->num_sms) != 0;
     }
     for (int s = 0; s < HIVIS_MAX_BATCH; ++s) {
         c->kv_upper[s] = 0;
@@ -318,6 +352,38 @@ static int prepare_rho(hivis_ctx* c, const void* resid, int R, cudaStream_t st) 
         CKL(c, launch_gemv_alu(c->dtype, PRO_PLAIN, EPI_QKV, a, st));
     }
     return HIVIS_OK;
+}
+
+// Split the cache rows of the longest listed sequence: `want` splits if possible, at least 32 rows
+// per split, never more splits than the partial buffers hold.
+static void plan_attention(const hivis_ctx* c, int max_rows, int want, int* chunk, int* nsplit) {
+    if (want > c->nsplit_cap) want = c->nsplit_cap;
+    if (want < 1) want = 1;
+    int ch = (max_rows + want - 1) / want;
+    ch = (ch + 31) / 32 * 32;
+    if (ch < 32) ch = 32;
+    *chunk = ch;
+    *nsplit = (max_rows + ch - 1) / ch;
+}
+
+static void fill_chain_args(hivis_ctx* c, ChainArgs* a) {
+    const hivis_config& g = c->cfg;
+    memset(a, 0, sizeof(*a));
+    a->ph[PH_FC] = {c->fc, g.d, 2 * g.d};
+    a->ph[PH_QKV] = {c->wqkv, c->qkvw, g.d};
+    a->ph[PH_O] = {c->wo, g.d, c->qw};
+    a->ph[PH_GU] = {c->wgu, 2 * g.ffn, g.d};
+    a->ph[PH_DOWN] = {c->wdown, g.d, g.ffn};
+    a->ph[PH_LM] = {c->lm_head, g.vocab, g.d};
+    a->d = g.d; a->qw = c->qw; a->kvw = c->kvw; a->F = g.ffn; a->V = g.vocab; a->Hq = g.n_q_heads;
+    a->Hkv = g.n_kv_heads; a->dh = g.head_dim; a->max_len = g.max_len; a->eps = g.rms_eps;
+    a->scale = 1.0f / sqrtf((float)g.head_dim);
+    a->norm1 = c->norm1; a->norm2 = c->norm2; a->bqkv = c->bqkv; a->embed = c->embed;
+    a->kv_len = c->kv_len; a->pend_feat = c->pend_feat; a->pend_id = c->pend_id;
+    a->u = c->u; a->qkv = c->qkv; a->attn = c->attn; a->y = c->y; a->act = c->act; a->feat = c->feat;
+    a->keys = c->keys; a->Kc = c->Kc; a->Vc = c->Vc; a->inv_freq = c->inv_freq;
+    a->part_acc = c->part_acc; a->part_ml = c->part_ml; a->counters = c->counters;
+    a->bar_counter = c->bar_counter; a->error_flag = c->error_flag;
 }
 
 static bool use_mma(const hivis_ctx* c, int B, bool prefill) {
@@ -462,10 +528,34 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
         rc = prepare_rho(c, resid, n_resid, st);
         if (rc) return rc;
     }
+    if (B == 1 && c->opt_chain && c->chain_ok) {
+        // one sequence: all k steps in one persistent cooperative kernel
+        ChainArgs a;
+        fill_chain_args(c, &a);
+        a.k = k;
+        a.rho = resid ? c->rho : nullptr;
+        a.n_resid = resid ? n_resid : 1;
+        a.slot = sl.slot[0];
+        a.forced = forced_ids;
+        a.logits_out = out_logits;
+        a.out_ids = out_ids;
+        plan_attention(c, max_rows, c->num_sms / g.n_q_heads, &a.attn_chunk, &a.attn_nsplit);
+        a.bar_base = c->bar_count_host;
+        CKP(c, CLS_CHAIN, st, launch_draft_chain(a, c->dtype, c->num_sms, st));
+        c->bar_count_host += (u64)c->num_sms * (u64)(chain_barriers_per_step() * k);
+        const int s0 = sl.slot[0];
+        c->kv_upper[s0] += k;
+        c->pending[s0] = false;
+        c->last_k[s0] = k;
+        c->tap_B = 1;
+        c->tap_mma = false;
+        return HIVIS_OK;
+    }
     CKP(c, CLS_OTHER, st, launch_draft_setup(sl, k, d, c->d_slots, c->d_pos0, c->kv_len, c->pend_feat, c->pend_id, c->feat,
                               c->feat_h, c->cur_id, c->keys, c->key_stride, st));
     const bool mma = use_mma(c, B, false);
-    const int nsplit = (max_rows + c->chunk - 1) / c->chunk;
+    int chunk = 0, nsplit = 0;
+    plan_attention(c, max_rows, (max_rows + c->chunk - 1) / c->chunk, &chunk, &nsplit);
     const int tiles1 = (d + HIVIS_MMA_TILE_ROWS - 1) / HIVIS_MMA_TILE_ROWS;
     const int bstep = mma ? 16 : B;
     for (int s = 0; s < k; ++s) {
@@ -492,7 +582,7 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
             memset(&a, 0, sizeof(a));
             a.qkv = c->qkv; a.ld = c->qkvw; a.Kc = c->Kc; a.Vc = c->Vc; a.slots = c->d_slots; a.pos0 = c->d_pos0;
             a.step = s; a.inv_freq = c->inv_freq; a.Hq = g.n_q_heads; a.Hkv = g.n_kv_heads; a.dh = g.head_dim;
-            a.max_len = g.max_len; a.B = B; a.scale = 1.0f / sqrtf((float)g.head_dim); a.chunk = c->chunk;
+            a.max_len = g.max_len; a.B = B; a.scale = 1.0f / sqrtf((float)g.head_dim); a.chunk = chunk;
             a.nsplit = nsplit; a.part_acc = c->part_acc; a.part_ml = c->part_ml; a.counters = c->counters;
             a.attn = c->attn; a.attn_h = c->attn_h;
             CKP(c, CLS_ATTN, st, launch_attention(c->dtype, a, st));
@@ -639,6 +729,31 @@ int hivis_read_kv(hivis_ctx* c, int slot, int row0, int n, float* out_k, float* 
     CKL(c, launch_read_kv(c->dtype, c->Kc, c->Vc, slot, row0, n, c->cfg.n_kv_heads, c->cfg.head_dim,
                           c->cfg.max_len, out_k, out_v, (cudaStream_t)stream));
     return HIVIS_OK;
+}
+
+int hivis_set_option(hivis_ctx* c, int option, int value) {
+    if (!c) return HIVIS_ERR_ARG;
+    if (option == HIVIS_OPT_CHAIN_KERNEL) {
+        c->opt_chain = value != 0;
+        return HIVIS_OK;
+    }
+    return fail(c, HIVIS_ERR_ARG, "unknown option %d", option);
+}
+
+int hivis_status(hivis_ctx* c, void* stream) {
+    if (!c) return HIVIS_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    int flag = 0;
+    CK(c, cudaMemcpyAsync(&flag, c->error_flag, sizeof(int), cudaMemcpyDeviceToHost, st));
+    CK(c, cudaStreamSynchronize(st));
+    if (flag == 0) return HIVIS_OK;
+    // a kernel gave up on a wait: bring the barrier bookkeeping back to a known state
+    CK(c, cudaMemsetAsync(c->bar_counter, 0, sizeof(u64), st));
+    CK(c, cudaMemsetAsync(c->error_flag, 0, sizeof(int), st));
+    CK(c, cudaMemsetAsync(c->counters, 0, (size_t)c->rows_cap * c->cfg.n_q_heads * sizeof(int), st));
+    CK(c, cudaStreamSynchronize(st));
+    c->bar_count_host = 0;
+    return fail(c, HIVIS_ERR_TIMEOUT, "a device-side wait ran out (code %d); results of that call are invalid", flag);
 }
 
 int hivis_profile_begin(hivis_ctx* c) {

@@ -85,6 +85,48 @@ struct AttnArgs {
 cudaError_t launch_attention(int dtype, const AttnArgs& a, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------
+// Persistent chain kernel (one sequence, all k steps in one cooperative launch).
+// ---------------------------------------------------------------------------------------------
+enum { PH_FC = 0, PH_QKV, PH_O, PH_GU, PH_DOWN, PH_LM, PH_COUNT };
+
+struct ChainPhase {
+    const void* W;        // [N][K], context dtype
+    int N, K;
+};
+
+struct ChainArgs {
+    ChainPhase ph[PH_COUNT];
+    int k;
+    int d, qw, kvw, F, V, Hq, Hkv, dh, max_len;
+    float eps, scale;
+    const void *norm1, *norm2, *bqkv, *embed;
+    const float* rho;          // [n_resid][d] fp32, nullable
+    int n_resid;
+    int slot;
+    int* kv_len;
+    const float* pend_feat;    // [slots][d]
+    const int* pend_id;
+    float *u, *qkv, *attn, *y, *act, *feat;
+    u64* keys;                 // [k]
+    const int* forced;         // [k], nullable
+    float* logits_out;         // [k][V], nullable
+    int32_t* out_ids;          // [k]
+    void *Kc, *Vc;
+    const double* inv_freq;
+    float *part_acc, *part_ml;
+    int* counters;
+    int attn_chunk, attn_nsplit;
+    u64* bar_counter;          // arrival counter of the grid barrier, only ever incremented
+    u64 bar_base;              // its value when this launch starts
+    int* error_flag;           // set non-zero by a kernel that gave up on a wait
+    int off_x, off_part, off_bar, off_misc;   // shared-memory layout, filled by the launcher
+};
+// shared memory the kernel needs for these dimensions on `grid` CTAs; 0 = does not fit
+size_t chain_smem_bytes(const ChainArgs& a, int dtype, int grid);
+cudaError_t launch_draft_chain(ChainArgs& a, int dtype, int grid, cudaStream_t st);
+int chain_barriers_per_step();
+
+// ---------------------------------------------------------------------------------------------
 // Small kernels: state set-up, prefill bookkeeping, verification, layout changes, taps.
 // ---------------------------------------------------------------------------------------------
 struct SlotList {

@@ -1,6 +1,6 @@
 // Small kernels around the hot path: per-call state set-up, prefill bookkeeping, greedy
 // verification with KV rollback, layout changes at init, debug read-back.
-#include "hivis_internal.cuh"
+#include "attn_body.cuh"
 
 // ------------------------------------------------------------------------------------------
 // draft set-up / finish
@@ -124,9 +124,8 @@ __global__ void kv_append_kernel(const float* kv, const int* slot_of, const int*
     const float* v = k + kvw;
     for (int i = threadIdx.x; i < Hkv * half; i += blockDim.x) {
         const int h = i / half, e = i % half;
-        double sn, cs;
-        sincos((double)row * inv_freq[e], &sn, &cs);
-        const float c = (float)cs, s = (float)sn;
+        float c, s;
+        rope_cs(row, inv_freq[e], c, s);
         const float x0 = k[h * dh + e], x1 = k[h * dh + e + half];
         const long long o = (((long long)slot * Hkv + h) * max_len + row) * dh;
         store_from_float<WT>(Kc, o + e, x0 * c - x1 * s);

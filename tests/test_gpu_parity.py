@@ -32,6 +32,50 @@ def test_c1_ids_exact_and_tight_logits():
         case.close()
 
 
+@pytest.mark.parametrize("name", ["c1_tiny_f32_b1", "mini_mha_b1"])
+def test_chain_kernel_and_stepwise_kernels_agree(name):
+    """One sequence: the persistent chain kernel and the per-step kernels compute the same thing."""
+    wl = hi.workload(name)
+    case = Case(wl)
+    try:
+        case.drafter.set_chain_kernel(False)
+        res_step = check_draft_parity(case)
+        case.gpu_restore()
+        ids_s, logits_s = case.gpu_draft(forced=res_step["ids_o"])
+        case.drafter.set_chain_kernel(True)
+        case.gpu_restore()
+        ids_c, logits_c = case.gpu_draft(forced=res_step["ids_o"])
+        case.drafter.status()
+        assert row_rel_err(logits_c, logits_s).max() < 1e-4
+        check_kv_parity(case, res_step["ref"])
+    finally:
+        case.close()
+
+
+@pytest.mark.parametrize("T,k", [(300, 8), (1, 2), (64, 1)])
+def test_chain_kernel_long_and_short(T, k):
+    wl = hi.scaled(hi.workload("mini_mha_b1"), text_len=T, k=k, seed=4000 + T)
+    case = Case(wl)
+    try:
+        res = check_draft_parity(case)
+        case.drafter.status()
+        check_kv_parity(case, res["ref"])
+    finally:
+        case.close()
+
+
+def test_chain_kernel_gqa_b1():
+    wl = hi.scaled(hi.workload("mini_gqa_b3"), batch=1, k=4)
+    case = Case(wl)
+    try:
+        res = check_draft_parity(case)
+        case.drafter.status()
+        check_kv_parity(case, res["ref"])
+        check_verify_parity(case, res["ids_o"])
+    finally:
+        case.close()
+
+
 def test_intermediate_taps_match_oracle():
     wl = hi.workload("mini_mha_b5_ragged")
     case = Case(wl)
