@@ -206,6 +206,28 @@ int64_t hivis_launch_count(const hivis_ctx* ctx);
 
 const char* hivis_last_error(const hivis_ctx* ctx);
 
+/* Greedy verification that allocates nothing and needs no context.  (The paper has no counterpart:
+ * this is the arithmetic of hivis_verify offered to callers that cannot obtain device memory, such
+ * as a plug-in inside a server whose memory pool already owns the GPU, or code that runs after its
+ * host has closed the allocation phase.)  The per-row argmax keys live in a fixed array inside the
+ * library image, HIVIS_MAX_BATCH * (HIVIS_MAX_K + 1) 8-byte entries (8.5 KB) on every GPU that
+ * loads the library, held until the process exits.  The call uses no cudaMalloc, cudaFree or other
+ * allocating routine.
+ *   draft_ids [B, k] int32, target_logits [B, k+1, vocab] in logits_dtype: as for hivis_verify.
+ *   rows_before (nullable, int32 [B]): cache rows each sequence held before its draft; when given,
+ *   out_kv_len[b] = rows_before[b] + 1 + min(n, k-1), the row count hivis_verify would roll the
+ *   slot back to.  rows_before and out_kv_len are given together or both NULL.
+ *   out_accept, out_next: as for hivis_verify.  No library state is read or changed.
+ * The first call made with a given device current looks up the array's address on that device;
+ * make that first call outside any stream capture.  All calls on one device share the array and
+ * it keeps the previous call's contents (each call clears the part it uses on `stream` first), so
+ * two calls whose work overlaps on the GPU, e.g. on different streams, race: order them.
+ * Errors: CAPACITY (B > HIVIS_MAX_BATCH or k > HIVIS_MAX_K: the fixed array is too small), SHAPE,
+ * DTYPE, ARG, CUDA; the text is available from hivis_last_error(NULL).                           */
+int hivis_verify_noalloc(int B, int k, int vocab, const int32_t* draft_ids, const void* target_logits,
+                         int logits_dtype, const int32_t* rows_before, int32_t* out_accept,
+                         int32_t* out_next, int32_t* out_kv_len, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

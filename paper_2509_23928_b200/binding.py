@@ -17,7 +17,7 @@ ERRORS = {0: "OK", -1: "ARG", -2: "SHAPE", -3: "DTYPE", -4: "STATE", -5: "CAPACI
 EXPORTS = ("hivis_init", "hivis_destroy", "hivis_prefill", "hivis_draft", "hivis_verify", "hivis_reset",
            "hivis_get_kv_len", "hivis_set_kv_len", "hivis_read_kv", "hivis_debug_tap", "hivis_step_bytes",
            "hivis_launch_count", "hivis_last_error", "hivis_profile_begin", "hivis_profile_end", "hivis_set_option",
-           "hivis_status")
+           "hivis_status", "hivis_verify_noalloc")
 HIVIS_OPT_CHAIN_KERNEL = 0
 PROFILE_CLASSES = ("fuse_fc", "qkv", "attention", "o_proj", "gate_up", "down", "lm_head_argmax", "setup_finish",
                    "draft_chain")
@@ -70,6 +70,7 @@ def _load() -> C.CDLL:
     L.hivis_status.argtypes = [vp, vp]
     L.hivis_profile_begin.argtypes = [vp]
     L.hivis_profile_end.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int64)]
+    L.hivis_verify_noalloc.argtypes = [i32, i32, i32, vp, vp, i32, vp, vp, vp, vp, vp]
     L.hivis_last_error.argtypes = [vp]
     L.hivis_last_error.restype = C.c_char_p
     for n in EXPORTS:
@@ -139,6 +140,15 @@ def hivis_verify(ctx, B, seq_slots, k, draft_ids, target_logits, logits_dtype, o
     _check(lib.hivis_verify(ctx, int(B), _ints(seq_slots), int(k), _ptr(draft_ids), _ptr(target_logits),
                             int(logits_dtype), _ptr(out_accept), _ptr(out_next), _ptr(out_kv_len),
                             _stream(stream)), ctx)
+
+
+def hivis_verify_noalloc(B, k, vocab, draft_ids, target_logits, logits_dtype, rows_before, out_accept,
+                         out_next, out_kv_len=None, stream=None):
+    """Context-free greedy verification for callers that must not allocate device memory: the
+    argmax keys sit in a fixed array inside the library (at most 64 sequences, k <= 16)."""
+    _check(lib.hivis_verify_noalloc(int(B), int(k), int(vocab), _ptr(draft_ids), _ptr(target_logits),
+                                    int(logits_dtype), _ptr(rows_before), _ptr(out_accept), _ptr(out_next),
+                                    _ptr(out_kv_len), _stream(stream)))
 
 
 def hivis_reset(ctx, slot, stream=None):

@@ -90,6 +90,8 @@ static int fail(hivis_ctx* c, int code, const char* fmt, ...) {
     return code;
 }
 static char g_init_err[256] = "";
+// text for failures of calls that have no context; hivis_last_error(NULL) returns it
+void hivis_set_global_error(const char* msg) { snprintf(g_init_err, sizeof(g_init_err), "%s", msg); }
 
 #define CK(c, call)                                                                            \
     do {                                                                                       \
