@@ -19,6 +19,7 @@ EXPORTS = ("hivis_init", "hivis_destroy", "hivis_prefill", "hivis_draft", "hivis
            "hivis_launch_count", "hivis_last_error", "hivis_profile_begin", "hivis_profile_end", "hivis_set_option",
            "hivis_status", "hivis_verify_noalloc")
 HIVIS_OPT_CHAIN_KERNEL = 0
+HIVIS_OPT_TC_KERNEL = 1
 PROFILE_CLASSES = ("fuse_fc", "qkv", "attention", "o_proj", "gate_up", "down", "lm_head_argmax", "setup_finish",
                    "draft_chain")
 
@@ -283,6 +284,9 @@ class Drafter:
 
     def set_chain_kernel(self, on: bool):
         hivis_set_option(self.ctx, HIVIS_OPT_CHAIN_KERNEL, 1 if on else 0)
+
+    def set_tc_kernel(self, on: bool):
+        hivis_set_option(self.ctx, HIVIS_OPT_TC_KERNEL, 1 if on else 0)
 
     def status(self):
         hivis_status(self.ctx)

@@ -36,10 +36,19 @@ struct hivis_ctx {
     // persistent chain kernel
     int num_sms;
     bool chain_ok;                // cooperative launch available and the kernel fits
+    bool chain_ok_coop;           // cooperative launch available
     bool opt_chain;               // option HIVIS_OPT_CHAIN_KERNEL
     u64* bar_counter;
     u64 bar_count_host;           // value of *bar_counter once everything enqueued has run
     int* error_flag;
+    // tensor-core chain kernel (bf16, up to 16 sequences)
+    bool tc_ok;                   // cooperative launch available, shapes supported, tensor maps built
+    bool opt_tc;                  // option HIVIS_OPT_TC_KERNEL
+    TcMaps tc_maps;
+    float* tc_partial;
+    int* tile_ctr;
+    int tc_tiles;
+    bf16* zero_row;
     int *slot_of, *row_of;
     long long map_cap;
     // host mirrors
@@ -236,6 +245,11 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
     if (c->nsplit_cap > 64) c->nsplit_cap = 64;
     c->opt_chain = true;
     c->chain_ok = false;
+    c->opt_tc = true;
+    c->tc_ok = false;
+    c->tc_partial = nullptr;
+    c->tile_ctr = nullptr;
+    c->tc_tiles = 0;
     c->bar_count_host = 0;
     {
         int coop = 0;
@@ -246,6 +260,7 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
             coop = 0;
         }
         c->chain_ok = coop != 0 && c->num_sms > 0;
+        c->chain_ok_coop = c->chain_ok;
     }
     c->key_stride = cfg->max_k + 1;
     c->map_cap = MB * (long long)cfg->max_len;
@@ -273,7 +288,7 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
          dalloc(c, &c->part_ml, R * cfg->n_q_heads * (long long)c->nsplit_cap * 2) &&
          dalloc(c, &c->counters, R * cfg->n_q_heads) && dalloc(c, &c->bar_counter, 1) &&
          dalloc(c, &c->error_flag, 1) && dalloc(c, &c->slot_of, c->map_cap) &&
-         dalloc(c, &c->row_of, c->map_cap);
+         dalloc(c, &c->row_of, c->map_cap) && dalloc(c, &c->zero_row, d);
     if (!ok) {
         free_all(c);
         delete c;
@@ -314,6 +329,12 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
         CK(c, cudaMemsetAsync(c->counters, 0, R * cfg->n_q_heads * sizeof(int), st));
         CK(c, cudaMemsetAsync(c->bar_counter, 0, sizeof(u64), st));
         CK(c, cudaMemsetAsync(c->error_flag, 0, sizeof(int), st));
+        CK(c, cudaMemsetAsync(c->zero_row, 0, d * sizeof(bf16), st));
+        CK(c, cudaMemsetAsync(c->feat_h, 0, R * d * sizeof(bf16), st));
+        CK(c, cudaMemsetAsync(c->xq, 0, R * d * sizeof(bf16), st));
+        CK(c, cudaMemsetAsync(c->attn_h, 0, R * c->qw * sizeof(bf16), st));
+        CK(c, cudaMemsetAsync(c->xm, 0, R * d * sizeof(bf16), st));
+        CK(c, cudaMemsetAsync(c->act_h, 0, R * F * sizeof(bf16), st));
         CK(c, cudaMemsetAsync(c->Kc, 0, MB * c->kvw * (long long)cfg->max_len * es, st));
         CK(c, cudaMemsetAsync(c->Vc, 0, MB * c->kvw * (long long)cfg->max_len * es, st));
         return HIVIS_OK;
@@ -329,6 +350,19 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
         ChainArgs ca;
         fill_chain_args(c, &ca);
         c->chain_ok = chain_smem_bytes(ca, c->dtype, c->num_sms) != 0;
+    }
+    if (c->dtype == HIVIS_BF16 && c->num_sms > 0 && c->chain_ok_coop &&
+        tc_supported(cfg->d, cfg->head_dim, cfg->n_q_heads, cfg->n_kv_heads, cfg->ffn)) {
+        ChainArgs ca;
+        fill_chain_args(c, &ca);
+        c->tc_tiles = tc_max_tiles(ca.ph);
+        bool ok2 = dalloc(c, &c->tc_partial, (size_t)c->num_sms * 2 * 16 * 128) && dalloc(c, &c->tile_ctr, c->tc_tiles);
+        if (ok2) ok2 = cudaMemsetAsync(c->tile_ctr, 0, c->tc_tiles * sizeof(int), st) == cudaSuccess;
+        if (ok2)
+            ok2 = tc_build_maps(&c->tc_maps, ca.ph, cfg->d, c->qw, cfg->ffn, cfg->vocab, c->embed, c->feat_h, c->xq,
+                                c->attn_h, c->xm, c->act_h, c->zero_row) == cudaSuccess;
+        if (!ok2) cudaGetLastError();
+        c->tc_ok = ok2;
     }
     for (int s = 0; s < HIVIS_MAX_BATCH; ++s) {
         c->kv_upper[s] = 0;
@@ -529,6 +563,48 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
     if (resid) {
         rc = prepare_rho(c, resid, n_resid, st);
         if (rc) return rc;
+    }
+    if (c->tc_ok && c->opt_tc && B <= 16) {
+        // bf16, up to 16 sequences: all k steps in one cooperative tensor-core kernel
+        const int lo = B <= 8 ? 1 : 0;
+        CKP(c, CLS_OTHER, st, launch_tc_setup(sl, k, d, lo, c->d_slots, c->d_pos0, c->kv_len, c->pend_feat, c->pend_id,
+                                              c->feat, c->feat_h, c->cur_id, c->keys, c->key_stride, st));
+        ChainArgs ca;
+        fill_chain_args(c, &ca);
+        TcArgs a;
+        memset(&a, 0, sizeof(a));
+        for (int p = 0; p < PH_COUNT; ++p) a.ph[p] = ca.ph[p];
+        a.k = k; a.B = B; a.lo = lo;
+        a.d = d; a.qw = c->qw; a.kvw = c->kvw; a.F = F; a.V = V; a.Hq = g.n_q_heads; a.Hkv = g.n_kv_heads;
+        a.dh = g.head_dim; a.max_len = g.max_len; a.eps = g.rms_eps; a.scale = 1.0f / sqrtf((float)g.head_dim);
+        a.norm1 = (const bf16*)c->norm1; a.norm2 = (const bf16*)c->norm2; a.bqkv = (const bf16*)c->bqkv;
+        a.rho = resid ? c->rho : nullptr; a.n_resid = resid ? n_resid : 1;
+        a.slots = c->d_slots; a.pos0 = c->d_pos0; a.cur_id = c->cur_id; a.forced = forced_ids;
+        a.keys = c->keys; a.key_stride = c->key_stride;
+        a.u = c->u; a.qkv = c->qkv; a.attn = c->attn; a.y = c->y; a.feat = c->feat;
+        a.feat_h = c->feat_h; a.xq_h = c->xq; a.attn_h = c->attn_h; a.xm_h = c->xm; a.act_h = c->act_h;
+        a.ssq1 = c->ssq1; a.ssq2 = c->ssq2; a.logits_out = out_logits;
+        a.partial = c->tc_partial; a.tile_ctr = c->tile_ctr;
+        a.Kc = c->Kc; a.Vc = c->Vc; a.inv_freq = c->inv_freq; a.part_acc = c->part_acc; a.part_ml = c->part_ml;
+        a.counters = c->counters;
+        {
+            const int gq = (g.n_q_heads / g.n_kv_heads) % 7 == 0 ? 7 : 1;
+            const int groups = B * (g.n_q_heads / gq);
+            plan_attention(c, max_rows, (c->num_sms + groups - 1) / groups, &a.attn_chunk, &a.attn_nsplit);
+        }
+        a.bar_counter = c->bar_counter; a.bar_base = c->bar_count_host; a.error_flag = c->error_flag;
+        CKP(c, CLS_CHAIN, st, launch_tc_chain(c->tc_maps, a, c->num_sms, st));
+        c->bar_count_host += (u64)c->num_sms * (u64)(tc_barriers_per_step() * k);
+        CKP(c, CLS_OTHER, st, launch_draft_finish(B, k, c->keys, c->key_stride, out_ids, st));
+        for (int b = 0; b < B; ++b) {
+            const int s = sl.slot[b];
+            c->kv_upper[s] += k;
+            c->pending[s] = false;
+            c->last_k[s] = k;
+        }
+        c->tap_B = B;
+        c->tap_mma = true;
+        return HIVIS_OK;
     }
     if (B == 1 && c->opt_chain && c->chain_ok) {
         // one sequence: all k steps in one persistent cooperative kernel
@@ -739,6 +815,10 @@ int hivis_set_option(hivis_ctx* c, int option, int value) {
         c->opt_chain = value != 0;
         return HIVIS_OK;
     }
+    if (option == HIVIS_OPT_TC_KERNEL) {
+        c->opt_tc = value != 0;
+        return HIVIS_OK;
+    }
     return fail(c, HIVIS_ERR_ARG, "unknown option %d", option);
 }
 
@@ -753,6 +833,7 @@ int hivis_status(hivis_ctx* c, void* stream) {
     CK(c, cudaMemsetAsync(c->bar_counter, 0, sizeof(u64), st));
     CK(c, cudaMemsetAsync(c->error_flag, 0, sizeof(int), st));
     CK(c, cudaMemsetAsync(c->counters, 0, (size_t)c->rows_cap * c->cfg.n_q_heads * sizeof(int), st));
+    if (c->tile_ctr) CK(c, cudaMemsetAsync(c->tile_ctr, 0, (size_t)c->tc_tiles * sizeof(int), st));
     CK(c, cudaStreamSynchronize(st));
     c->bar_count_host = 0;
     return fail(c, HIVIS_ERR_TIMEOUT, "a device-side wait ran out (code %d); results of that call are invalid", flag);

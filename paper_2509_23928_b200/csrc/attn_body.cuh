@@ -22,13 +22,30 @@ __device__ __forceinline__ void rope_cs(int pos, double inv_freq, float& c, floa
     sincosf((float)r, &s, &c);
 }
 
-template <typename WT, int DH, int GQ, int NW>
+// Barrier among the NT threads that work on a unit: the whole CTA (BAR == 0) or a named barrier.
+template <int BAR, int NT>
+__device__ __forceinline__ void attn_sync() {
+    if (BAR == 0) __syncthreads();
+    else asm volatile("bar.sync %0, %1;" ::"r"(BAR), "r"(NT) : "memory");
+}
+
+// bf16 copy of an attention output element; with lo_rows > 0 the rounding remainder goes to row
+// b + lo_rows, so that a bf16 tensor-core operand carries the value to about 16 mantissa bits.
+__device__ __forceinline__ void attn_store_h(const AttnArgs& a, int b, int qw, int col, float o) {
+    if (!a.attn_h) return;
+    const bf16 hi = __float2bfloat16_rn(o);
+    a.attn_h[(long long)b * qw + col] = hi;
+    if (a.lo_rows > 0) a.attn_h[(long long)(b + a.lo_rows) * qw + col] = __float2bfloat16_rn(o - __bfloat162float(hi));
+}
+
+// `tid` is the caller's index among the NW*32 threads that take part (0-based).
+template <typename WT, int DH, int GQ, int NW, int BAR = 0>
 __device__ __forceinline__ void attn_unit(const AttnArgs& a, int split, int hg, int b, int p, int slot,
-                                          AttnSmem<NW, GQ, DH>& sm) {
+                                          AttnSmem<NW, GQ, DH>& sm, int tid = threadIdx.x) {
     constexpr int EPL = DH / 32;                     // head-dim elements per lane in the PV phase
     constexpr int NT = NW * 32;
     constexpr int VEC = 16 / (int)sizeof(WT);
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int warp = tid >> 5, lane = tid & 31;
     const int G = a.Hq / a.Hkv;
     const int h0 = hg * GQ;                          // first query head of this unit
     const int kvh = h0 / G;
@@ -42,7 +59,7 @@ __device__ __forceinline__ void attn_unit(const AttnArgs& a, int split, int hg, 
     const int qw = a.Hq * DH, kvw = a.Hkv * DH;
     const float* qkv = a.qkv + (long long)b * a.ld;
 
-    __syncthreads();                                 // the previous unit's readers are done with sm
+    attn_sync<BAR, NT>();                                 // the previous unit's readers are done with sm
     for (int i = tid; i < GQ * half; i += NT) {
         const int gq = i / half, j = i % half;
         float c, s;
@@ -78,7 +95,7 @@ __device__ __forceinline__ void attn_unit(const AttnArgs& a, int split, int hg, 
             sm.vnew[j] = v;
         }
     }
-    __syncthreads();
+    attn_sync<BAR, NT>();
 
     float m_run[GQ], l_run[GQ], acc[GQ][EPL];
 #pragma unroll
@@ -198,7 +215,7 @@ __device__ __forceinline__ void attn_unit(const AttnArgs& a, int split, int hg, 
 #pragma unroll
         for (int e = 0; e < EPL; ++e) sm.acc_s[warp][gq][lane * EPL + e] = acc[gq][e];
     }
-    __syncthreads();
+    attn_sync<BAR, NT>();
     const bool single = nsplits == 1;
     for (int i = tid; i < GQ * DH; i += NT) {
         const int gq = i / DH, dd = i % DH;
@@ -216,7 +233,7 @@ __device__ __forceinline__ void attn_unit(const AttnArgs& a, int split, int hg, 
         if (single) {
             const float o = A / L;
             a.attn[(long long)b * qw + h * DH + dd] = o;
-            if (a.attn_h) a.attn_h[(long long)b * qw + h * DH + dd] = __float2bfloat16_rn(o);
+            attn_store_h(a, b, qw, h * DH + dd, o);
         } else {
             const long long pi = ((long long)b * a.Hq + h) * a.nsplit + split;
             a.part_acc[pi * DH + dd] = A;
@@ -229,14 +246,14 @@ __device__ __forceinline__ void attn_unit(const AttnArgs& a, int split, int hg, 
     if (single) return;
     // arrival counter: the last unit of this (sequence, head group) merges the splits; nobody waits
     __threadfence();
-    __syncthreads();
+    attn_sync<BAR, NT>();
     if (tid == 0) {
         int* ctr = a.counters + (long long)b * a.Hq + h0;
         const int old = atomicAdd(ctr, 1);
         sm.s_last = (old == nsplits - 1);
         if (sm.s_last) *ctr = 0;
     }
-    __syncthreads();
+    attn_sync<BAR, NT>();
     if (!sm.s_last) return;
     __threadfence();
     for (int i = tid; i < GQ * DH; i += NT) {
@@ -253,6 +270,6 @@ __device__ __forceinline__ void attn_unit(const AttnArgs& a, int split, int hg, 
         }
         const float o = A / L;
         a.attn[(long long)b * qw + h * DH + dd] = o;
-        if (a.attn_h) a.attn_h[(long long)b * qw + h * DH + dd] = __float2bfloat16_rn(o);
+        attn_store_h(a, b, qw, h * DH + dd, o);
     }
 }

@@ -81,6 +81,7 @@ struct AttnArgs {
     int* counters;        // [B][Hq] arrival counters, zero between launches
     float* attn;          // [B][Hq*dh] fp32
     bf16* attn_h;         // [B][Hq*dh] bf16 copy
+    int lo_rows;          // > 0: rounding remainders of attn_h go to rows b + lo_rows
 };
 cudaError_t launch_attention(int dtype, const AttnArgs& a, cudaStream_t st);
 
@@ -126,9 +127,6 @@ size_t chain_smem_bytes(const ChainArgs& a, int dtype, int grid);
 cudaError_t launch_draft_chain(ChainArgs& a, int dtype, int grid, cudaStream_t st);
 int chain_barriers_per_step();
 
-// ---------------------------------------------------------------------------------------------
-// Small kernels: state set-up, prefill bookkeeping, verification, layout changes, taps.
-// ---------------------------------------------------------------------------------------------
 struct SlotList {
     int n;
     int slot[HIVIS_MAX_BATCH];
@@ -136,6 +134,64 @@ struct SlotList {
 struct CuSeqlens {
     int v[HIVIS_MAX_BATCH + 1];
 };
+
+// ---------------------------------------------------------------------------------------------
+// Tensor-core chain kernel (bf16 weights, 1..16 sequences): all k steps in one cooperative launch,
+// weights streamed by TMA into a shared-memory ring, tcgen05.mma with the weights as the M operand
+// (128 rows) and the batch as N (16 columns), accumulators in tensor memory.
+// ---------------------------------------------------------------------------------------------
+#define TC_OP_ROWS 16          // rows of every bf16 operand buffer that the tensor maps cover
+enum { TCM_W = 0,              // PH_COUNT weight maps, box 64 x 128
+       TCM_X_FEAT = PH_COUNT, TCM_X_XQ, TCM_X_ATTN, TCM_X_XM, TCM_X_ACT,   // operand maps, box 64 x 16
+       TCM_EMBED,              // embedding table, box 64 x 1 (one row per copy)
+       TCM_ZERO,               // one row of zeros, box 64 x 1
+       TCM_COUNT };
+struct TcMaps {
+    alignas(64) unsigned char m[TCM_COUNT][128];     // CUtensorMap objects
+};
+struct TcArgs {
+    ChainPhase ph[PH_COUNT];
+    int k, B;
+    int lo;                    // 1: B <= 8, operand rows [B, 2B) carry the bf16 rounding remainders
+    int d, qw, kvw, F, V, Hq, Hkv, dh, max_len;
+    float eps, scale;
+    const bf16 *norm1, *norm2, *bqkv;
+    const float* rho;          // [n_resid][d] fp32, nullable
+    int n_resid;
+    const int *slots, *pos0, *cur_id;     // [B]
+    const int* forced;         // [B][k], nullable
+    u64* keys;                 // [B][key_stride]
+    int key_stride;
+    float *u, *qkv, *attn, *y, *feat;     // fp32 activations [B][width]
+    bf16 *feat_h, *xq_h, *attn_h, *xm_h, *act_h;   // bf16 operands [TC_OP_ROWS][width]
+    float *ssq1, *ssq2;        // [tiles*4][16] partial sums of squares of u / y
+    float* logits_out;         // [B][k][V], nullable
+    float* partial;            // [grid*2][16][128] split-tile partial accumulators
+    int* tile_ctr;             // arrival counters of split tiles, zero between phases
+    void *Kc, *Vc;
+    const double* inv_freq;
+    float *part_acc, *part_ml;
+    int* counters;
+    int attn_chunk, attn_nsplit;
+    u64* bar_counter;
+    u64 bar_base;
+    int* error_flag;
+};
+// fills `maps` for the given buffers; returns cudaSuccess or an error (driver entry point missing, bad shape)
+cudaError_t tc_build_maps(TcMaps* maps, const ChainPhase* ph, int d, int qw, int F, int V, const void* embed,
+                          const bf16* feat_h, const bf16* xq_h, const bf16* attn_h, const bf16* xm_h,
+                          const bf16* act_h, const bf16* zero_row);
+bool tc_supported(int d, int dh, int Hq, int Hkv, int F);
+int tc_max_tiles(const ChainPhase* ph);
+cudaError_t launch_tc_chain(const TcMaps& maps, const TcArgs& a, int grid, cudaStream_t st);
+cudaError_t launch_tc_setup(const SlotList& sl, int k, int d, int lo, int* d_slots, int* d_pos0, int* kv_len,
+                            const float* pend_feat, const int* pend_id, float* feat, bf16* feat_h,
+                            int* cur_id, u64* keys, int key_stride, cudaStream_t st);
+int tc_barriers_per_step();
+
+// ---------------------------------------------------------------------------------------------
+// Small kernels: state set-up, prefill bookkeeping, verification, layout changes, taps.
+// ---------------------------------------------------------------------------------------------
 
 // draft set-up: slots -> device, pos0 = kv_len[slot], feat = pending feature, ids = pending id;
 // clears the argmax keys [B][k]; advances kv_len by k.

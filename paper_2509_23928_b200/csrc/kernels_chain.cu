@@ -283,7 +283,7 @@ __global__ void __launch_bounds__(CHAIN_THREADS, 1) draft_chain_kernel(const Cha
     aa.qkv = a.qkv; aa.ld = a.qw + 2 * a.kvw; aa.Kc = a.Kc; aa.Vc = a.Vc; aa.slots = nullptr; aa.pos0 = nullptr;
     aa.step = 0; aa.inv_freq = a.inv_freq; aa.Hq = a.Hq; aa.Hkv = a.Hkv; aa.dh = a.dh; aa.max_len = a.max_len;
     aa.B = 1; aa.scale = a.scale; aa.chunk = a.attn_chunk; aa.nsplit = a.attn_nsplit; aa.part_acc = a.part_acc;
-    aa.part_ml = a.part_ml; aa.counters = a.counters; aa.attn = a.attn; aa.attn_h = nullptr;
+    aa.part_ml = a.part_ml; aa.counters = a.counters; aa.attn = a.attn; aa.attn_h = nullptr; aa.lo_rows = 0;
 
     for (int s = 0; s < a.k && alive; ++s) {
         // ============================================================ fusion FC + residual

@@ -1,0 +1,797 @@
+// Tensor-core draft-chain kernel: all k chained draft steps of up to 16 sequences in ONE cooperative
+// launch, bf16 weights.
+//
+// One CTA per SM, 8 warps with fixed roles:
+//   warp 0 (one thread)  producer: streams weight tiles (128 rows x 64 k, 16 KB) and the matching batch
+//                        operand tiles (16 rows x 64 k, 2 KB) into a shared-memory ring with TMA
+//                        (cp.async.bulk.tensor, 128-byte swizzle, mbarrier complete_tx).  Weight tiles do
+//                        not depend on activations, so their loads run ahead through phase and step
+//                        boundaries; only the operand tile of a stage waits for the grid barrier.
+//   warp 1 (one thread)  issues tcgen05.mma (M = 128 weight rows, N = 16 batch columns, K = 16, four per
+//                        stage), accumulating in tensor memory (two 16-column accumulators, so the next
+//                        tile's MMAs overlap the previous tile's epilogue); tcgen05.commit frees stages.
+//   warps 4-7            epilogue: tcgen05.ld (one weight row per thread, 16 batch values), then the fused
+//                        output stage of the phase (residuals, RMSNorm statistics and gains, RoPE-free
+//                        QKV bias, SiLU*up, LM-head argmax keys) and the bf16 operand of the next phase.
+//   warps 2-7            split-KV attention over the text-only cache between the QKV and O phases.
+//
+// Work split: a phase with T row tiles and KB k-blocks is T*KB tile-k-blocks, laid out tile-major and cut
+// into equal contiguous ranges, one per CTA (so every SM streams the same number of bytes whatever the
+// matrix shape).  A tile that straddles CTAs is finished by whichever contributor arrives last: everyone
+// writes its partial accumulator to global scratch and bumps the tile's arrival counter; the last one adds
+// the partials in contributor order (fixed, so results do not depend on timing) and runs the output stage.
+// Nobody waits for anybody inside a phase.
+//
+// Batch operand: activations are rounded to bf16 for the MMA; for B <= 8 the rounding remainder is fed
+// through the unused columns (rows [B, 2B) of every operand buffer) and added in the output stage, which
+// keeps about 16 mantissa bits of the activations.
+//
+// Every wait is bounded.  A wait that runs out raises the error flag and poisons the CTA: all roles then
+// run through their remaining schedule without waiting, issuing no further copies or MMAs, so that named
+// barriers still pair up, tensor memory is freed and the kernel returns.
+#include <cuda.h>
+
+#include "attn_body.cuh"
+
+#define TC_THREADS 256
+#define TC_STAGES 10
+#define TC_BK 64
+#define TC_TM 128
+#define TC_TN 16
+#define TC_A_BYTES (TC_TM * TC_BK * 2)
+#define TC_B_BYTES (TC_TN * TC_BK * 2)
+#define TC_ATT_WARPS 6
+#define TC_ATT_THREADS (TC_ATT_WARPS * 32)
+#define TC_EPI_THREADS 128
+#define TC_BAR_ATT 2
+#define TC_BAR_EPI 3
+#define TC_WAIT_CYCLES 2000000000ll      // ~1 s: far beyond any legitimate wait
+#define TC_TMEM_COLS 32
+
+// instruction descriptor of tcgen05.mma kind::f16: fp32 accumulate, bf16 x bf16, both K-major, N=16, M=128
+#define TC_IDESC ((1u << 4) | (1u << 7) | (1u << 10) | ((TC_TN >> 3) << 17) | ((TC_TM >> 4) << 24))
+
+namespace {
+
+struct TcParams {
+    TcMaps maps;
+    TcArgs a;
+};
+
+struct TcCtl {
+    u64 full[TC_STAGES], empty[TC_STAGES], tfull[2], tempty[2];
+    uint32_t tmem_base;
+    int abort_flag;
+    int last_flag;
+    float scale[16];
+    float red[8][16];
+};
+
+__device__ __forceinline__ uint32_t saddr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ u64 policy_evict_first() {
+    u64 pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ u64 policy_evict_last() {
+    u64 pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+// 2-D tiled TMA load: box of the tensor map at element coordinates (x = inner, y = row)
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* map, int x, int y, uint32_t bar, u64 pol) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%2, %3}], [%4], %5;" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(bar), "l"(pol)
+        : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, u64 adesc, u64 bdesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"((uint32_t)TC_IDESC), "r"(accumulate)
+        : "memory");
+}
+// shared-memory matrix descriptor: K-major tile whose rows are 128 bytes, 128-byte swizzle, 8-row groups
+// 1024 bytes apart
+__device__ __forceinline__ u64 tc_smem_desc(uint32_t addr) {
+    const uint32_t lo = ((addr >> 4) & 0x3FFFu) | (1u << 16);
+    const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+    return ((u64)hi << 32) | lo;
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ u64 ld_acquire_u64(const u64* p) {
+    u64 v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void red_release_add_u64(u64* p, u64 v) {
+    asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ int ld_relaxed_int(const int* p) {
+    int v;
+    asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
+
+// ---- bounded waits -------------------------------------------------------------------------------
+__device__ __forceinline__ bool poisoned(const TcCtl* ctl) { return *(volatile const int*)&ctl->abort_flag != 0; }
+__device__ __forceinline__ void poison(TcCtl* ctl, int* error_flag, int code) {
+    atomicCAS(error_flag, 0, code);
+    *(volatile int*)&ctl->abort_flag = 1;
+}
+__device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, TcCtl* ctl, int* error_flag, int code) {
+    if (poisoned(ctl)) return false;
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    unsigned it = 0;
+    while (!mbar_try(bar, parity)) {
+        if ((++it & 63u) == 0u) {
+            if (poisoned(ctl)) return false;
+            if (ld_relaxed_int(error_flag) != 0) { *(volatile int*)&ctl->abort_flag = 1; return false; }
+            if (clock64() - t0 > TC_WAIT_CYCLES) { poison(ctl, error_flag, code); return false; }
+        }
+    }
+    return true;
+}
+// wait until the grid-wide arrival counter reaches `target`
+__device__ __forceinline__ bool wait_grid(const u64* counter, u64 target, TcCtl* ctl, int* error_flag, int code) {
+    if (poisoned(ctl)) return false;
+    const long long t0 = clock64();
+    unsigned it = 0;
+    while (ld_acquire_u64(counter) < target) {
+        if ((++it & 63u) == 0u) {
+            if (poisoned(ctl)) return false;
+            if (ld_relaxed_int(error_flag) != 0) { *(volatile int*)&ctl->abort_flag = 1; return false; }
+            if (clock64() - t0 > TC_WAIT_CYCLES) { poison(ctl, error_flag, code); return false; }
+        }
+    }
+    return true;
+}
+
+// ---- schedule --------------------------------------------------------------------------------------
+// grid barriers of one step, in order: after FC, QKV, attention, O, gate/up, down, LM head
+#define TC_BARS_PER_STEP 7
+__device__ __forceinline__ int need_seq(int step, int p) {                              // barrier its operand needs (-1: none)
+    if (p == PH_FC) return step == 0 ? -1 : (step - 1) * TC_BARS_PER_STEP + 6;
+    if (p == PH_QKV) return step * TC_BARS_PER_STEP + 0;
+    return step * TC_BARS_PER_STEP + p;              // O needs attention (2), GU needs O (3), DOWN 4, LM 5
+}
+struct PhaseShape {
+    int nkb, ntiles;
+    long long W;
+};
+__device__ __forceinline__ PhaseShape phase_shape(const TcArgs& a, int p) {
+    PhaseShape s;
+    s.nkb = (a.ph[p].K + TC_BK - 1) / TC_BK;
+    s.ntiles = (a.ph[p].N + TC_TM - 1) / TC_TM;
+    s.W = (long long)s.nkb * s.ntiles;
+    return s;
+}
+__device__ __forceinline__ long long range_lo(long long W, int c, int G) { return W * c / G; }
+// CTA whose range contains tile-k-block `idx`
+__device__ __forceinline__ int owner_of(long long W, int G, long long idx) {
+    int c = (int)(idx * G / W);
+    if (c >= G) c = G - 1;
+    while (c + 1 < G && range_lo(W, c + 1, G) <= idx) ++c;
+    while (c > 0 && range_lo(W, c, G) > idx) --c;
+    return c;
+}
+
+// cursor over one CTA's tile-k-blocks through all phases and steps
+struct Cursor {
+    int step, p;
+    long long idx, hi;
+    int nkb;
+    bool live;
+};
+__device__ __forceinline__ void cursor_enter(Cursor& c, const TcArgs& a, int cta, int G) {
+    // position on the first non-empty phase range at or after (step, p)
+    while (c.live) {
+        const PhaseShape s = phase_shape(a, c.p);
+        c.idx = range_lo(s.W, cta, G);
+        c.hi = range_lo(s.W, cta + 1, G);
+        c.nkb = s.nkb;
+        if (c.idx < c.hi) return;
+        if (++c.p == PH_COUNT) {
+            c.p = 0;
+            if (++c.step == a.k) c.live = false;
+        }
+    }
+}
+__device__ __forceinline__ void cursor_next(Cursor& c, const TcArgs& a, int cta, int G) {
+    if (++c.idx < c.hi) return;
+    if (++c.p == PH_COUNT) {
+        c.p = 0;
+        if (++c.step == a.k) { c.live = false; return; }
+    }
+    cursor_enter(c, a, cta, G);
+}
+
+// ---- producer ------------------------------------------------------------------------------------
+__device__ void tc_producer(const TcParams& P, TcCtl* ctl, uint32_t smemA, uint32_t smemB, int cta, int G) {
+    const TcArgs& a = P.a;
+    const u64 pol_w = policy_evict_first(), pol_x = policy_evict_last();
+    Cursor ca{0, 0, 0, 0, 0, true}, cb{0, 0, 0, 0, 0, true};
+    cursor_enter(ca, a, cta, G);
+    cursor_enter(cb, a, cta, G);
+    unsigned a_cnt = 0, b_cnt = 0;
+    u64 seen = 0;
+    int ids[16];
+    int ids_step = -1;
+    const int dkb = a.d / TC_BK;
+    long long t0 = clock64();
+    while (ca.live || b_cnt < a_cnt) {
+        bool progress = false;
+        if (poisoned(ctl)) break;
+        if (ca.live) {
+            const unsigned slot = a_cnt % TC_STAGES, use = a_cnt / TC_STAGES;
+            if (use == 0 || mbar_test(saddr(&ctl->empty[slot]), (use - 1) & 1u)) {
+                const uint32_t bar = saddr(&ctl->full[slot]);
+                mbar_expect_tx(bar, TC_A_BYTES + TC_B_BYTES);
+                const int tile = (int)(ca.idx / ca.nkb), kb = (int)(ca.idx % ca.nkb);
+                tma_load_2d(smemA + slot * TC_A_BYTES, &P.maps.m[TCM_W + ca.p], kb * TC_BK, tile * TC_TM, bar, pol_w);
+                cursor_next(ca, a, cta, G);
+                ++a_cnt;
+                progress = true;
+            }
+        }
+        if (b_cnt < a_cnt) {
+            const int need = need_seq(cb.step, cb.p);
+            bool ready = need < 0;
+            if (!ready) {
+                const u64 target = a.bar_base + (u64)G * (u64)(need + 1);
+                if (seen < target) seen = ld_acquire_u64(a.bar_counter);
+                if (seen >= target) {
+                    ready = true;
+                }
+            }
+            if (ready) {
+                const unsigned slot = b_cnt % TC_STAGES;
+                const uint32_t bar = saddr(&ctl->full[slot]);
+                const uint32_t dst = smemB + slot * TC_B_BYTES;
+                const int kb = (int)(cb.idx % cb.nkb);
+                if (cb.p == PH_FC && kb >= dkb) {
+                    // embedding half of the fusion FC: one row per copy, gathered by token id
+                    if (ids_step != cb.step) {
+                        fence_proxy_async_all();
+                        for (int b = 0; b < a.B; ++b) {
+                            if (cb.step == 0) ids[b] = __ldcg(a.cur_id + b);
+                            else if (a.forced) ids[b] = __ldcg(a.forced + (long long)b * a.k + (cb.step - 1));
+                            else ids[b] = key_index(__ldcg(a.keys + (long long)b * a.key_stride + (cb.step - 1)));
+                            if (ids[b] < 0 || ids[b] >= a.V) ids[b] = 0;
+                        }
+                        ids_step = cb.step;
+                    }
+                    const int x = (kb - dkb) * TC_BK;
+#pragma unroll 1
+                    for (int r = 0; r < TC_TN; ++r) {
+                        if (r < a.B) tma_load_2d(dst + r * 128, &P.maps.m[TCM_EMBED], x, ids[r], bar, pol_x);
+                        else tma_load_2d(dst + r * 128, &P.maps.m[TCM_ZERO], 0, 0, bar, pol_x);
+                    }
+                } else {
+                    int m = TCM_X_FEAT;
+                    if (cb.p == PH_QKV) m = TCM_X_XQ;
+                    else if (cb.p == PH_O) m = TCM_X_ATTN;
+                    else if (cb.p == PH_GU) m = TCM_X_XM;
+                    else if (cb.p == PH_DOWN) m = TCM_X_ACT;
+                    fence_proxy_async_all();
+                    tma_load_2d(dst, &P.maps.m[m], kb * TC_BK, 0, bar, pol_x);
+                }
+                cursor_next(cb, a, cta, G);
+                ++b_cnt;
+                progress = true;
+            }
+        }
+        if (progress) {
+            t0 = clock64();
+        } else {
+            if (ld_relaxed_int(a.error_flag) != 0) { *(volatile int*)&ctl->abort_flag = 1; break; }
+            if (clock64() - t0 > TC_WAIT_CYCLES) { poison(ctl, a.error_flag, 3); break; }
+        }
+    }
+    if (poisoned(ctl)) {
+        // copies already issued still land in this CTA's shared memory: give them time before the CTA exits
+        for (unsigned i = b_cnt > TC_STAGES ? b_cnt - TC_STAGES : 0; i < b_cnt; ++i) {
+            const uint32_t bar = saddr(&ctl->full[i % TC_STAGES]);
+            const long long t1 = clock64();
+            while (!mbar_test(bar, (i / TC_STAGES) & 1u))
+                if (clock64() - t1 > 20000000ll) break;
+        }
+        const long long t1 = clock64();
+        while (clock64() - t1 < 2000000ll) {}
+    }
+}
+
+// ---- MMA issuer ----------------------------------------------------------------------------------
+__device__ void tc_mma_issuer(const TcParams& P, TcCtl* ctl, uint32_t smemA, uint32_t smemB, int cta, int G) {
+    const TcArgs& a = P.a;
+    const uint32_t tmem = ctl->tmem_base;
+    unsigned seg_cnt = 0, c_cnt = 0;
+    for (int s = 0; s < a.k; ++s)
+        for (int p = 0; p < PH_COUNT; ++p) {
+            const PhaseShape sh = phase_shape(a, p);
+            long long idx = range_lo(sh.W, cta, G);
+            const long long hi = range_lo(sh.W, cta + 1, G);
+            while (idx < hi) {
+                const int kb0 = (int)(idx % sh.nkb);
+                const int n = (int)((hi - idx) < (long long)(sh.nkb - kb0) ? (hi - idx) : (long long)(sh.nkb - kb0));
+                const unsigned acc = seg_cnt & 1u, use = seg_cnt >> 1;
+                if (use > 0) wait_mbar(saddr(&ctl->tempty[acc]), (use - 1) & 1u, ctl, a.error_flag, 4);
+                tc_fence_after();
+                for (int j = 0; j < n; ++j) {
+                    const unsigned slot = c_cnt % TC_STAGES;
+                    const bool ok = wait_mbar(saddr(&ctl->full[slot]), (c_cnt / TC_STAGES) & 1u, ctl, a.error_flag, 5);
+                    if (ok) {
+                        tc_fence_after();
+                        const u64 ad = tc_smem_desc(smemA + slot * TC_A_BYTES);
+                        const u64 bd = tc_smem_desc(smemB + slot * TC_B_BYTES);
+#pragma unroll
+                        for (int kk = 0; kk < TC_BK / 16; ++kk)
+                            tc_mma(tmem + acc * TC_TN, ad + (u64)(kk * 2), bd + (u64)(kk * 2), (j > 0 || kk > 0) ? 1u : 0u);
+                        tc_commit(saddr(&ctl->empty[slot]));
+                    }
+                    ++c_cnt;
+                }
+                if (!poisoned(ctl)) tc_commit(saddr(&ctl->tfull[acc]));
+                ++seg_cnt;
+                idx += n;
+            }
+        }
+}
+
+// ---- output stages ---------------------------------------------------------------------------------
+__device__ __forceinline__ void store_operand(bf16* buf, int width, int b, int col, float x, int lo_rows) {
+    const bf16 hi = __float2bfloat16_rn(x);
+    buf[(long long)b * width + col] = hi;
+    if (lo_rows > 0) buf[(long long)(b + lo_rows) * width + col] = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+
+// per-sequence scale 1/rms recovered from the partial sums of squares of the producing phase
+__device__ __forceinline__ void epi_compute_scales(const TcArgs& a, TcCtl* ctl, const float* ssq, int etid) {
+    const int entries = ((a.d + TC_TM - 1) / TC_TM) * 4;
+    const int b = etid & 15, part = etid >> 4;
+    float t = 0.f;
+    for (int i = part; i < entries; i += 8) t += __ldcg(ssq + (long long)i * 16 + b);
+    ctl->red[part][b] = t;
+    named_sync(TC_BAR_EPI, TC_EPI_THREADS);
+    if (etid < 16) {
+        float tot = 0.f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) tot += ctl->red[q][etid];
+        ctl->scale[etid] = rsqrtf(tot / (float)a.d + a.eps);
+    }
+    named_sync(TC_BAR_EPI, TC_EPI_THREADS);
+}
+
+__device__ void epi_output(const TcArgs& a, TcCtl* ctl, int p, int s, int tile, const float (&v)[16], int w4, int lane) {
+    const int N = a.ph[p].N;
+    const int row = tile * TC_TM + w4 * 32 + lane;
+    const bool rok = row < N;
+    const int B = a.B;
+    const int lo_rows = a.lo ? B : 0;
+    float val[16];
+#pragma unroll
+    for (int b = 0; b < 16; ++b) val[b] = 0.f;
+#pragma unroll
+    for (int b = 0; b < 16; ++b)
+        if (b < B) val[b] = v[b] + ((a.lo && b + B < 16) ? v[(b + B) & 15] : 0.f);
+
+    if (p == PH_FC || p == PH_O) {
+        const float* rho = (p == PH_FC && a.rho) ? a.rho + (long long)(s < a.n_resid - 1 ? s : a.n_resid - 1) * a.d : nullptr;
+        const bf16* gamma = p == PH_FC ? a.norm1 : a.norm2;
+        float* outf = p == PH_FC ? a.u : a.y;
+        bf16* outh = p == PH_FC ? a.xq_h : a.xm_h;
+        float* ssq = p == PH_FC ? a.ssq1 : a.ssq2;
+        const float g = rok ? __bfloat162float(gamma[row]) : 0.f;
+        const float add0 = (rok && rho) ? rho[row] : 0.f;
+#pragma unroll
+        for (int b = 0; b < 16; ++b) {
+            if (b >= B) break;
+            float r = 0.f;
+            if (rok) {
+                r = val[b] + (p == PH_FC ? add0 : __ldcg(a.u + (long long)b * N + row));
+                outf[(long long)b * N + row] = r;
+                store_operand(outh, N, b, row, g * r, lo_rows);
+            }
+            float sq = r * r;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+            if (lane == 0) ssq[(long long)(tile * 4 + w4) * 16 + b] = sq;
+        }
+    } else if (p == PH_QKV) {
+        const float bias = (rok && a.bqkv) ? __bfloat162float(a.bqkv[row]) : 0.f;
+        if (rok) {
+#pragma unroll
+            for (int b = 0; b < 16; ++b) {
+                if (b >= B) break;
+                a.qkv[(long long)b * N + row] = val[b] * ctl->scale[b] + bias;
+            }
+        }
+    } else if (p == PH_GU) {
+        // even rows are gate_i, odd rows up_i (i = row / 2): adjacent lanes exchange their values
+        const int F = N >> 1;
+#pragma unroll
+        for (int b = 0; b < 16; ++b) {
+            if (b >= B) break;
+            const float mine = val[b] * ctl->scale[b];
+            const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
+            if (rok && ((b & 1) == (lane & 1))) {
+                const float gate = (lane & 1) ? other : mine, up = (lane & 1) ? mine : other;
+                const float act = gate / (1.f + expf(-gate)) * up;
+                store_operand(a.act_h, F, b, row >> 1, act, lo_rows);
+            }
+        }
+    } else if (p == PH_DOWN) {
+        if (rok) {
+#pragma unroll
+            for (int b = 0; b < 16; ++b) {
+                if (b >= B) break;
+                const float r = __ldcg(a.y + (long long)b * N + row) + val[b];
+                a.feat[(long long)b * N + row] = r;
+                store_operand(a.feat_h, N, b, row, r, lo_rows);
+            }
+        }
+    } else {   // PH_LM
+#pragma unroll
+        for (int b = 0; b < 16; ++b) {
+            if (b >= B) break;
+            if (rok && a.logits_out) a.logits_out[((long long)b * a.k + s) * a.V + row] = val[b];
+            u64 key = rok ? pack_key(val[b], row) : 0ull;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const u64 other = __shfl_xor_sync(0xffffffffu, key, o);
+                key = other > key ? other : key;
+            }
+            if (lane == 0 && key) atomicMax(a.keys + (long long)b * a.key_stride + s, key);
+        }
+    }
+}
+
+// ---- epilogue warps: GEMM phases -------------------------------------------------------------------
+// Runs phase p of step s for this CTA's range and arrives on the phase's grid barrier.
+__device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, unsigned& seg_cnt, int cta, int G,
+                                  int w4, int lane) {
+    const TcArgs& a = P.a;
+    const int etid = w4 * 32 + lane;
+    const PhaseShape sh = phase_shape(a, p);
+    const long long lo = range_lo(sh.W, cta, G), hi = range_lo(sh.W, cta + 1, G);
+    long long idx = lo;
+    bool need_scale = (p == PH_QKV || p == PH_GU);
+    while (idx < hi) {
+        const int tile = (int)(idx / sh.nkb), kb0 = (int)(idx % sh.nkb);
+        const int n = (int)((hi - idx) < (long long)(sh.nkb - kb0) ? (hi - idx) : (long long)(sh.nkb - kb0));
+        const unsigned acc = seg_cnt & 1u;
+        wait_mbar(saddr(&ctl->tfull[acc]), (seg_cnt >> 1) & 1u, ctl, a.error_flag, 6);
+        tc_fence_after();
+        float v[16];
+        tc_ld16(ctl->tmem_base + ((uint32_t)(w4 * 32) << 16) + acc * TC_TN, v);
+        tc_fence_before();
+        mbar_arrive(saddr(&ctl->tempty[acc]));
+        ++seg_cnt;
+        if (need_scale) {       // the operand of this phase has arrived, so the producing phase is complete
+            epi_compute_scales(a, ctl, p == PH_QKV ? a.ssq1 : a.ssq2, etid);
+            need_scale = false;
+        }
+        bool finish = true;
+        if (!(kb0 == 0 && n == sh.nkb)) {
+            // a tile shared with other CTAs: publish the partial accumulator; the last arriver finishes the tile
+            float* mine = a.partial + (long long)(cta * 2 + (idx == lo ? 0 : 1)) * (16 * TC_TM);
+#pragma unroll
+            for (int c = 0; c < 16; ++c) mine[c * TC_TM + etid] = v[c];
+            __threadfence();
+            named_sync(TC_BAR_EPI, TC_EPI_THREADS);
+            if (etid == 0) {
+                // contributors = the CTAs whose (non-empty) ranges meet this tile, in range order
+                const long long t0 = (long long)tile * sh.nkb;
+                int nc = 0;
+                for (long long i = t0; i < t0 + sh.nkb; ++nc) i = range_lo(sh.W, owner_of(sh.W, G, i) + 1, G);
+                const int old = atomicAdd(a.tile_ctr + tile, 1);
+                const int last = old == nc - 1;
+                if (last) a.tile_ctr[tile] = 0;
+                ctl->last_flag = last;
+            }
+            named_sync(TC_BAR_EPI, TC_EPI_THREADS);
+            finish = ctl->last_flag != 0;
+            if (finish) {
+                __threadfence();
+                const long long t0 = (long long)tile * sh.nkb;
+#pragma unroll
+                for (int c = 0; c < 16; ++c) v[c] = 0.f;
+                for (long long i = t0; i < t0 + sh.nkb;) {
+                    const int cc = owner_of(sh.W, G, i);
+                    const float* src = a.partial + (long long)(cc * 2 + (i == range_lo(sh.W, cc, G) ? 0 : 1)) * (16 * TC_TM);
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) v[c] += __ldcg(src + c * TC_TM + etid);
+                    i = range_lo(sh.W, cc + 1, G);
+                }
+            }
+            named_sync(TC_BAR_EPI, TC_EPI_THREADS);      // last_flag may be rewritten by the next segment
+        }
+        if (finish) epi_output(a, ctl, p, s, tile, v, w4, lane);
+        idx += n;
+    }
+    // This CTA's part of the phase is done: arrive on the grid barrier.  All arrivals are counted in one
+    // counter, so a CTA may arrive for this phase only once the barrier before it is complete.  With work in
+    // the phase that is implied (its operand tiles were loaded after that barrier); without work, wait for it.
+    __threadfence();
+    named_sync(TC_BAR_EPI, TC_EPI_THREADS);
+    if (etid == 0) {
+        const int need = need_seq(s, p);
+        if (lo == hi && need >= 0)
+            wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(need + 1), ctl, a.error_flag, 8);
+        fence_proxy_async_all();
+        red_release_add_u64(a.bar_counter, 1ull);
+    }
+}
+
+}  // namespace
+
+template <int DH, int GQ>
+__global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_constant__ TcParams P) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    const TcArgs& a = P.a;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int cta = blockIdx.x, G = gridDim.x;
+    unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const uint32_t smemA = saddr(smem);
+    const uint32_t smemB = smemA + TC_STAGES * TC_A_BYTES;
+    TcCtl* ctl = (TcCtl*)(smem + TC_STAGES * (TC_A_BYTES + TC_B_BYTES));
+    typedef AttnSmem<TC_ATT_WARPS, GQ, DH> ASm;
+    ASm* asm_ = (ASm*)(smem + TC_STAGES * (TC_A_BYTES + TC_B_BYTES) + ((sizeof(TcCtl) + 127) & ~(size_t)127));
+
+    if (tid == 0) {
+        for (int i = 0; i < TC_STAGES; ++i) {
+            mbar_init(saddr(&ctl->full[i]), 1);
+            mbar_init(saddr(&ctl->empty[i]), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(saddr(&ctl->tfull[i]), 1);
+            mbar_init(saddr(&ctl->tempty[i]), TC_EPI_THREADS);
+        }
+        ctl->abort_flag = 0;
+        ctl->last_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async_all();
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(saddr(&ctl->tmem_base)),
+                     "r"((uint32_t)TC_TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    if (warp == 0) {
+        if (lane == 0) tc_producer(P, ctl, smemA, smemB, cta, G);
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) tc_mma_issuer(P, ctl, smemA, smemB, cta, G);
+        __syncwarp();
+    } else {
+        // warps 2..7: attention; warps 4..7 also the epilogue of every GEMM phase
+        const int atid = tid - 64;
+        const int w4 = warp - 4;
+        const bool is_epi = warp >= 4;
+        unsigned seg_cnt = 0;
+        AttnArgs aa;
+        aa.qkv = a.qkv; aa.ld = a.qw + 2 * a.kvw; aa.Kc = a.Kc; aa.Vc = a.Vc; aa.slots = a.slots; aa.pos0 = a.pos0;
+        aa.step = 0; aa.inv_freq = a.inv_freq; aa.Hq = a.Hq; aa.Hkv = a.Hkv; aa.dh = a.dh; aa.max_len = a.max_len;
+        aa.B = a.B; aa.scale = a.scale; aa.chunk = a.attn_chunk; aa.nsplit = a.attn_nsplit; aa.part_acc = a.part_acc;
+        aa.part_ml = a.part_ml; aa.counters = a.counters; aa.attn = a.attn; aa.attn_h = a.attn_h;
+        aa.lo_rows = a.lo ? a.B : 0;
+        const int hgroups = a.Hq / GQ;
+        const int nunits = a.B * hgroups * a.attn_nsplit;
+        for (int s = 0; s < a.k; ++s) {
+            if (is_epi) {
+                tc_epilogue_phase(P, ctl, s, PH_FC, seg_cnt, cta, G, w4, lane);
+                tc_epilogue_phase(P, ctl, s, PH_QKV, seg_cnt, cta, G, w4, lane);
+            }
+            // ---- attention: needs every CTA's QKV rows
+            if (atid == 0)
+                wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(s * TC_BARS_PER_STEP + 2), ctl, a.error_flag, 7);
+            named_sync(TC_BAR_ATT, TC_ATT_THREADS);
+            if (!poisoned(ctl)) {
+                for (int unit = cta; unit < nunits; unit += G) {
+                    const int split = unit % a.attn_nsplit;
+                    const int rest = unit / a.attn_nsplit;
+                    const int hg = rest % hgroups, b = rest / hgroups;
+                    attn_unit<bf16, DH, GQ, TC_ATT_WARPS, TC_BAR_ATT>(aa, split, hg, b, __ldg(a.pos0 + b) + s,
+                                                                      __ldg(a.slots + b), *asm_, atid);
+                }
+            }
+            __threadfence();
+            named_sync(TC_BAR_ATT, TC_ATT_THREADS);
+            if (atid == 0) {
+                fence_proxy_async_all();
+                red_release_add_u64(a.bar_counter, 1ull);
+            }
+            if (is_epi) {
+                tc_epilogue_phase(P, ctl, s, PH_O, seg_cnt, cta, G, w4, lane);
+                tc_epilogue_phase(P, ctl, s, PH_GU, seg_cnt, cta, G, w4, lane);
+                tc_epilogue_phase(P, ctl, s, PH_DOWN, seg_cnt, cta, G, w4, lane);
+                tc_epilogue_phase(P, ctl, s, PH_LM, seg_cnt, cta, G, w4, lane);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(ctl->tmem_base), "r"((uint32_t)TC_TMEM_COLS)
+                     : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------ set-up kernel
+__global__ void tc_setup_kernel(SlotList sl, int k, int d, int lo, int* d_slots, int* d_pos0, int* kv_len,
+                                const float* pend_feat, const int* pend_id, float* feat, bf16* feat_h, int* cur_id,
+                                u64* keys, int key_stride) {
+    const int b = blockIdx.x, slot = sl.slot[b];
+    if (threadIdx.x == 0) {
+        d_slots[b] = slot;
+        const int rows = kv_len[slot];
+        d_pos0[b] = rows;
+        kv_len[slot] = rows + k;            // every draft step appends one K/V row
+        cur_id[b] = pend_id[slot];
+    }
+    if (threadIdx.x < k) keys[(long long)b * key_stride + threadIdx.x] = 0ull;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        const float v = pend_feat[(long long)slot * d + i];
+        feat[(long long)b * d + i] = v;
+        const bf16 hi = __float2bfloat16_rn(v);
+        feat_h[(long long)b * d + i] = hi;
+        if (lo) feat_h[(long long)(b + sl.n) * d + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
+    }
+}
+cudaError_t launch_tc_setup(const SlotList& sl, int k, int d, int lo, int* d_slots, int* d_pos0, int* kv_len,
+                            const float* pend_feat, const int* pend_id, float* feat, bf16* feat_h, int* cur_id,
+                            u64* keys, int key_stride, cudaStream_t st) {
+    tc_setup_kernel<<<sl.n, 256, 0, st>>>(sl, k, d, lo, d_slots, d_pos0, kv_len, pend_feat, pend_id, feat, feat_h,
+                                          cur_id, keys, key_stride);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// bf16 row-major [rows][cols] matrix, box = box_rows x 64 columns, 128-byte swizzle, zero fill outside
+static cudaError_t encode_map(unsigned char* out, const void* base, long long rows, long long cols, int box_rows,
+                              CUtensorMapL2promotion promo) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return cudaErrorNotSupported;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {TC_BK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn((CUtensorMap*)out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides,
+                          box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, promo,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+bool tc_supported(int d, int dh, int Hq, int Hkv, int F) {
+    return d % TC_BK == 0 && (dh == 64 || dh == 128) && Hkv > 0 && Hq % Hkv == 0 && F % 8 == 0;
+}
+
+int tc_max_tiles(const ChainPhase* ph) {
+    int m = 0;
+    for (int p = 0; p < PH_COUNT; ++p) {
+        const int t = (ph[p].N + TC_TM - 1) / TC_TM;
+        if (t > m) m = t;
+    }
+    return m;
+}
+
+int tc_barriers_per_step() { return TC_BARS_PER_STEP; }
+
+cudaError_t tc_build_maps(TcMaps* maps, const ChainPhase* ph, int d, int qw, int F, int V, const void* embed,
+                          const bf16* feat_h, const bf16* xq_h, const bf16* attn_h, const bf16* xm_h,
+                          const bf16* act_h, const bf16* zero_row) {
+    static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
+    cudaError_t e;
+    for (int p = 0; p < PH_COUNT; ++p) {
+        e = encode_map(maps->m[TCM_W + p], ph[p].W, ph[p].N, ph[p].K, TC_TM, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+        if (e != cudaSuccess) return e;
+    }
+    const struct { int idx; const bf16* base; int cols; } ops[5] = {
+        {TCM_X_FEAT, feat_h, d}, {TCM_X_XQ, xq_h, d}, {TCM_X_ATTN, attn_h, qw}, {TCM_X_XM, xm_h, d}, {TCM_X_ACT, act_h, F}};
+    for (int i = 0; i < 5; ++i) {
+        e = encode_map(maps->m[ops[i].idx], ops[i].base, TC_OP_ROWS, ops[i].cols, TC_TN, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+        if (e != cudaSuccess) return e;
+    }
+    e = encode_map(maps->m[TCM_EMBED], embed, V, d, 1, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+    if (e != cudaSuccess) return e;
+    return encode_map(maps->m[TCM_ZERO], zero_row, 1, d, 1, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+}
+
+template <int DH, int GQ>
+static cudaError_t tc_launch_t(const TcParams& P, int grid, cudaStream_t st) {
+    static bool attr_set = false;
+    const size_t smem = 1024 + (size_t)TC_STAGES * (TC_A_BYTES + TC_B_BYTES) + ((sizeof(TcCtl) + 127) & ~(size_t)127) +
+                        sizeof(AttnSmem<TC_ATT_WARPS, GQ, DH>);
+    if (smem > 227 * 1024) return cudaErrorInvalidValue;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc_chain_kernel<DH, GQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    void* params[] = {(void*)&P};
+    return cudaLaunchCooperativeKernel((const void*)tc_chain_kernel<DH, GQ>, dim3(grid), dim3(TC_THREADS), params, smem, st);
+}
+
+cudaError_t launch_tc_chain(const TcMaps& maps, const TcArgs& a, int grid, cudaStream_t st) {
+    TcParams P;
+    P.maps = maps;
+    P.a = a;
+    const int G = a.Hq / a.Hkv;
+    const int gq = (G % 7 == 0) ? 7 : 1;
+    if (a.dh == 128) return gq == 7 ? tc_launch_t<128, 7>(P, grid, st) : tc_launch_t<128, 1>(P, grid, st);
+    return gq == 7 ? tc_launch_t<64, 7>(P, grid, st) : tc_launch_t<64, 1>(P, grid, st);
+}

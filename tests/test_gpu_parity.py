@@ -11,11 +11,16 @@ SMALL = ["c1_tiny_f32_b1", "mini_mha_b1", "mini_mha_b5_ragged", "mini_gqa_b16_ra
          "tiny_f32_b4_ragged"]
 
 
+@pytest.mark.parametrize("tc", [True, False])
 @pytest.mark.parametrize("name", SMALL)
-def test_draft_kv_verify_parity_small(name):
+def test_draft_kv_verify_parity_small(name, tc):
+    """tc=True: the persistent tensor-core kernel (bf16 workloads); tc=False: the per-step kernels
+    (and, for one sequence, the ALU chain kernel)."""
     case = Case(hi.workload(name))
     try:
+        case.drafter.set_tc_kernel(tc)
         res = check_draft_parity(case)
+        case.drafter.status()
         check_kv_parity(case, res["ref"])              # cache after the teacher-forced run = oracle's run
         check_verify_parity(case, res["ids_o"])
     finally:
@@ -38,6 +43,7 @@ def test_chain_kernel_and_stepwise_kernels_agree(name):
     wl = hi.workload(name)
     case = Case(wl)
     try:
+        case.drafter.set_tc_kernel(False)
         case.drafter.set_chain_kernel(False)
         res_step = check_draft_parity(case)
         case.gpu_restore()
@@ -52,11 +58,13 @@ def test_chain_kernel_and_stepwise_kernels_agree(name):
         case.close()
 
 
+@pytest.mark.parametrize("tc", [True, False])
 @pytest.mark.parametrize("T,k", [(300, 8), (1, 2), (64, 1)])
-def test_chain_kernel_long_and_short(T, k):
+def test_chain_kernel_long_and_short(T, k, tc):
     wl = hi.scaled(hi.workload("mini_mha_b1"), text_len=T, k=k, seed=4000 + T)
     case = Case(wl)
     try:
+        case.drafter.set_tc_kernel(tc)
         res = check_draft_parity(case)
         case.drafter.status()
         check_kv_parity(case, res["ref"])
@@ -64,10 +72,12 @@ def test_chain_kernel_long_and_short(T, k):
         case.close()
 
 
-def test_chain_kernel_gqa_b1():
+@pytest.mark.parametrize("tc", [True, False])
+def test_chain_kernel_gqa_b1(tc):
     wl = hi.scaled(hi.workload("mini_gqa_b3"), batch=1, k=4)
     case = Case(wl)
     try:
+        case.drafter.set_tc_kernel(tc)
         res = check_draft_parity(case)
         case.drafter.status()
         check_kv_parity(case, res["ref"])
@@ -76,10 +86,12 @@ def test_chain_kernel_gqa_b1():
         case.close()
 
 
-def test_intermediate_taps_match_oracle():
+@pytest.mark.parametrize("tc", [True, False])
+def test_intermediate_taps_match_oracle(tc):
     wl = hi.workload("mini_mha_b5_ragged")
     case = Case(wl)
     try:
+        case.drafter.set_tc_kernel(tc)
         case.gpu_prefill()
         case.gpu_draft(1)
         rho = case.oracle.fold_residuals(case.resid)
