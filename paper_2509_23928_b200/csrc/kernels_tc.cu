@@ -2,18 +2,20 @@
 // launch, bf16 weights.
 //
 // One CTA per SM, 8 warps with fixed roles:
-//   warp 0 (one thread)  producer: streams weight tiles (128 rows x 64 k, 16 KB) and the matching batch
-//                        operand tiles (16 rows x 64 k, 2 KB) into a shared-memory ring with TMA
-//                        (cp.async.bulk.tensor, 128-byte swizzle, mbarrier complete_tx).  Weight tiles do
-//                        not depend on activations, so their loads run ahead through phase and step
-//                        boundaries; only the operand tile of a stage waits for the grid barrier.
+//   warp 0 (one thread)  weight producer: streams weight tiles (128 rows x 64 k, 16 KB) into a shared-memory
+//                        ring with TMA (cp.async.bulk.tensor, 128-byte swizzle, mbarrier complete_tx).
+//                        Weight tiles do not depend on activations, so their loads run ahead through phase
+//                        and step boundaries, limited only by the ring.
+//   warp 2               operand producer: the matching batch-operand tiles (16 rows x 64 k, 2 KB) in the
+//                        same order; the first tile of a phase waits for the grid barrier before it.
 //   warp 1 (one thread)  issues tcgen05.mma (M = 128 weight rows, N = 16 batch columns, K = 16, four per
 //                        stage), accumulating in tensor memory (two 16-column accumulators, so the next
 //                        tile's MMAs overlap the previous tile's epilogue); tcgen05.commit frees stages.
 //   warps 4-7            epilogue: tcgen05.ld (one weight row per thread, 16 batch values), then the fused
 //                        output stage of the phase (residuals, RMSNorm statistics and gains, RoPE-free
 //                        QKV bias, SiLU*up, LM-head argmax keys) and the bf16 operand of the next phase.
-//   warps 2-7            split-KV attention over the text-only cache between the QKV and O phases.
+//                        Between the QKV and O phases the same warps run the split-KV attention over the
+//                        text-only cache.
 //
 // Work split: a phase with T row tiles and KB k-blocks is T*KB tile-k-blocks, laid out tile-major and cut
 // into equal contiguous ranges, one per CTA (so every SM streams the same number of bytes whatever the
@@ -40,10 +42,8 @@
 #define TC_TN 16
 #define TC_A_BYTES (TC_TM * TC_BK * 2)
 #define TC_B_BYTES (TC_TN * TC_BK * 2)
-#define TC_ATT_WARPS 6
-#define TC_ATT_THREADS (TC_ATT_WARPS * 32)
+#define TC_ATT_WARPS 4               // the epilogue warps also run the attention
 #define TC_EPI_THREADS 128
-#define TC_BAR_ATT 2
 #define TC_BAR_EPI 3
 #define TC_WAIT_CYCLES 2000000000ll      // ~1 s: far beyond any legitimate wait
 #define TC_TMEM_COLS 32
@@ -225,21 +225,26 @@ __device__ __forceinline__ int owner_of(long long W, int G, long long idx) {
     return c;
 }
 
-// cursor over one CTA's tile-k-blocks through all phases and steps
+// Cursor over one CTA's tile-k-blocks through all phases and steps.  Divisions happen only when a phase is
+// entered; stepping to the next k-block is a few integer instructions (the producers are single threads).
 struct Cursor {
     int step, p;
-    long long idx, hi;
-    int nkb;
-    bool live;
+    int tile, kb, left, nkb;
+    bool live, entered;         // entered: this k-block is the first of its phase for this CTA
 };
 __device__ __forceinline__ void cursor_enter(Cursor& c, const TcArgs& a, int cta, int G) {
     // position on the first non-empty phase range at or after (step, p)
     while (c.live) {
         const PhaseShape s = phase_shape(a, c.p);
-        c.idx = range_lo(s.W, cta, G);
-        c.hi = range_lo(s.W, cta + 1, G);
+        const long long lo = range_lo(s.W, cta, G), hi = range_lo(s.W, cta + 1, G);
         c.nkb = s.nkb;
-        if (c.idx < c.hi) return;
+        c.left = (int)(hi - lo);
+        if (c.left > 0) {
+            c.tile = (int)(lo / s.nkb);
+            c.kb = (int)(lo % s.nkb);
+            c.entered = true;
+            return;
+        }
         if (++c.p == PH_COUNT) {
             c.p = 0;
             if (++c.step == a.k) c.live = false;
@@ -247,7 +252,14 @@ __device__ __forceinline__ void cursor_enter(Cursor& c, const TcArgs& a, int cta
     }
 }
 __device__ __forceinline__ void cursor_next(Cursor& c, const TcArgs& a, int cta, int G) {
-    if (++c.idx < c.hi) return;
+    c.entered = false;
+    if (--c.left > 0) {
+        if (++c.kb == c.nkb) {
+            c.kb = 0;
+            ++c.tile;
+        }
+        return;
+    }
     if (++c.p == PH_COUNT) {
         c.p = 0;
         if (++c.step == a.k) { c.live = false; return; }
@@ -255,120 +267,106 @@ __device__ __forceinline__ void cursor_next(Cursor& c, const TcArgs& a, int cta,
     cursor_enter(c, a, cta, G);
 }
 
-// ---- producer ------------------------------------------------------------------------------------
-__device__ void tc_producer(const TcParams& P, TcCtl* ctl, uint32_t smemA, uint32_t smemB, int cta, int G) {
+// after a give-up: copies already issued still land in this CTA's shared memory; give them time
+__device__ __forceinline__ void drain_after_poison() {
+    const long long t1 = clock64();
+    while (clock64() - t1 < 4000000ll) {}
+}
+
+// ---- producers -------------------------------------------------------------------------------------
+// Weight tiles: arms the stage's barrier with the bytes of both tiles and issues the weight copy.  Runs
+// ahead of the grid barriers, limited only by the ring.
+__device__ void tc_producer_w(const TcParams& P, TcCtl* ctl, uint32_t smemA, int cta, int G) {
     const TcArgs& a = P.a;
-    const u64 pol_w = policy_evict_first(), pol_x = policy_evict_last();
-    Cursor ca{0, 0, 0, 0, 0, true}, cb{0, 0, 0, 0, 0, true};
-    cursor_enter(ca, a, cta, G);
-    cursor_enter(cb, a, cta, G);
-    unsigned a_cnt = 0, b_cnt = 0;
-    u64 seen = 0;
-    int ids[16];
-    int ids_step = -1;
+    const u64 pol_w = policy_evict_first();
+    Cursor c{0, 0, 0, 0, 0, 0, true, false};
+    cursor_enter(c, a, cta, G);
+    unsigned slot = 0, round = 0;
     const int dkb = a.d / TC_BK;
-    long long t0 = clock64();
-    while (ca.live || b_cnt < a_cnt) {
-        bool progress = false;
+    const int erows = a.lo ? 2 * a.B : a.B;
+    while (c.live) {
+        if (round > 0 && !wait_mbar(saddr(&ctl->empty[slot]), (round - 1) & 1u, ctl, a.error_flag, 3)) break;
         if (poisoned(ctl)) break;
-        if (ca.live) {
-            const unsigned slot = a_cnt % TC_STAGES, use = a_cnt / TC_STAGES;
-            if (use == 0 || mbar_test(saddr(&ctl->empty[slot]), (use - 1) & 1u)) {
-                const uint32_t bar = saddr(&ctl->full[slot]);
-                mbar_expect_tx(bar, TC_A_BYTES + TC_B_BYTES);
-                const int tile = (int)(ca.idx / ca.nkb), kb = (int)(ca.idx % ca.nkb);
-                tma_load_2d(smemA + slot * TC_A_BYTES, &P.maps.m[TCM_W + ca.p], kb * TC_BK, tile * TC_TM, bar, pol_w);
-                cursor_next(ca, a, cta, G);
-                ++a_cnt;
-                progress = true;
-            }
-        }
-        if (b_cnt < a_cnt) {
-            const int need = need_seq(cb.step, cb.p);
-            bool ready = need < 0;
-            if (!ready) {
-                const u64 target = a.bar_base + (u64)G * (u64)(need + 1);
-                if (seen < target) seen = ld_acquire_u64(a.bar_counter);
-                if (seen >= target) {
-                    ready = true;
-                }
-            }
-            if (ready) {
-                const unsigned slot = b_cnt % TC_STAGES;
-                const uint32_t bar = saddr(&ctl->full[slot]);
-                const uint32_t dst = smemB + slot * TC_B_BYTES;
-                const int kb = (int)(cb.idx % cb.nkb);
-                if (cb.p == PH_FC && kb >= dkb) {
-                    // embedding half of the fusion FC: one row per copy, gathered by token id
-                    if (ids_step != cb.step) {
-                        fence_proxy_async_all();
-                        for (int b = 0; b < a.B; ++b) {
-                            if (cb.step == 0) ids[b] = __ldcg(a.cur_id + b);
-                            else if (a.forced) ids[b] = __ldcg(a.forced + (long long)b * a.k + (cb.step - 1));
-                            else ids[b] = key_index(__ldcg(a.keys + (long long)b * a.key_stride + (cb.step - 1)));
-                            if (ids[b] < 0 || ids[b] >= a.V) ids[b] = 0;
-                        }
-                        ids_step = cb.step;
-                    }
-                    const int x = (kb - dkb) * TC_BK;
-#pragma unroll 1
-                    for (int r = 0; r < TC_TN; ++r) {
-                        if (r < a.B) tma_load_2d(dst + r * 128, &P.maps.m[TCM_EMBED], x, ids[r], bar, pol_x);
-                        else tma_load_2d(dst + r * 128, &P.maps.m[TCM_ZERO], 0, 0, bar, pol_x);
-                    }
-                } else {
-                    int m = TCM_X_FEAT;
-                    if (cb.p == PH_QKV) m = TCM_X_XQ;
-                    else if (cb.p == PH_O) m = TCM_X_ATTN;
-                    else if (cb.p == PH_GU) m = TCM_X_XM;
-                    else if (cb.p == PH_DOWN) m = TCM_X_ACT;
-                    fence_proxy_async_all();
-                    tma_load_2d(dst, &P.maps.m[m], kb * TC_BK, 0, bar, pol_x);
-                }
-                cursor_next(cb, a, cta, G);
-                ++b_cnt;
-                progress = true;
-            }
-        }
-        if (progress) {
-            t0 = clock64();
-        } else {
-            if (ld_relaxed_int(a.error_flag) != 0) { *(volatile int*)&ctl->abort_flag = 1; break; }
-            if (clock64() - t0 > TC_WAIT_CYCLES) { poison(ctl, a.error_flag, 3); break; }
-        }
+        const uint32_t bar = saddr(&ctl->full[slot]);
+        // the embedding half of the fusion FC brings only the operand rows in use (one 128-byte row per copy)
+        const uint32_t xbytes = (c.p == PH_FC && c.kb >= dkb) ? (uint32_t)erows * 128u : (uint32_t)TC_B_BYTES;
+        mbar_expect_tx(bar, TC_A_BYTES + xbytes);
+        tma_load_2d(smemA + slot * TC_A_BYTES, &P.maps.m[TCM_W + c.p], c.kb * TC_BK, c.tile * TC_TM, bar, pol_w);
+        cursor_next(c, a, cta, G);
+        if (++slot == TC_STAGES) { slot = 0; ++round; }
     }
-    if (poisoned(ctl)) {
-        // copies already issued still land in this CTA's shared memory: give them time before the CTA exits
-        for (unsigned i = b_cnt > TC_STAGES ? b_cnt - TC_STAGES : 0; i < b_cnt; ++i) {
-            const uint32_t bar = saddr(&ctl->full[i % TC_STAGES]);
-            const long long t1 = clock64();
-            while (!mbar_test(bar, (i / TC_STAGES) & 1u))
-                if (clock64() - t1 > 20000000ll) break;
+    if (poisoned(ctl)) drain_after_poison();
+}
+
+// Batch-operand tiles: same k-block order; the first tile of a phase waits for the grid barrier after
+// which the operand is complete.  Run by a whole warp with uniform control flow: lane 0 issues the tile
+// copies, and in the embedding half of the fusion FC lane r issues the copy of operand row r.
+__device__ void tc_producer_x(const TcParams& P, TcCtl* ctl, uint32_t smemB, int cta, int G, int lane) {
+    const TcArgs& a = P.a;
+    const u64 pol_x = policy_evict_last();
+    Cursor c{0, 0, 0, 0, 0, 0, true, false};
+    cursor_enter(c, a, cta, G);
+    unsigned slot = 0, round = 0;
+    int my_id = 0;
+    const int dkb = a.d / TC_BK;
+    const int erows = a.lo ? 2 * a.B : a.B;
+    int map_idx = TCM_X_FEAT;
+    while (c.live) {
+        if (c.entered) {
+            const int need = need_seq(c.step, c.p);
+            if (need >= 0) {
+                if (!wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(need + 1), ctl, a.error_flag, 9)) break;
+                // other CTAs wrote the operand through the generic proxy; TMA reads through the async proxy
+                fence_proxy_async_all();
+            }
+            if (c.p == PH_FC && lane < a.B) {
+                int id;
+                if (c.step == 0) id = __ldcg(a.cur_id + lane);
+                else if (a.forced) id = __ldcg(a.forced + (long long)lane * a.k + (c.step - 1));
+                else id = key_index(__ldcg(a.keys + (long long)lane * a.key_stride + (c.step - 1)));
+                my_id = (id < 0 || id >= a.V) ? 0 : id;
+            }
+            map_idx = c.p == PH_QKV ? TCM_X_XQ : c.p == PH_O ? TCM_X_ATTN : c.p == PH_GU ? TCM_X_XM
+                    : c.p == PH_DOWN ? TCM_X_ACT : TCM_X_FEAT;
         }
-        const long long t1 = clock64();
-        while (clock64() - t1 < 2000000ll) {}
+        if (round > 0 && !wait_mbar(saddr(&ctl->empty[slot]), (round - 1) & 1u, ctl, a.error_flag, 10)) break;
+        if (poisoned(ctl)) break;
+        const uint32_t bar = saddr(&ctl->full[slot]);
+        const uint32_t dst = smemB + slot * TC_B_BYTES;
+        if (c.p == PH_FC && c.kb >= dkb) {
+            // embedding half of the fusion FC: rows gathered by token id; remainder rows are zero
+            const int x = (c.kb - dkb) * TC_BK;
+            if (lane < a.B) tma_load_2d(dst + lane * 128, &P.maps.m[TCM_EMBED], x, my_id, bar, pol_x);
+            else if (lane < erows) tma_load_2d(dst + lane * 128, &P.maps.m[TCM_ZERO], 0, 0, bar, pol_x);
+        } else if (lane == 0) {
+            tma_load_2d(dst, &P.maps.m[map_idx], c.kb * TC_BK, 0, bar, pol_x);
+        }
+        __syncwarp();
+        cursor_next(c, a, cta, G);
+        if (++slot == TC_STAGES) { slot = 0; ++round; }
     }
+    __syncwarp();
+    if (poisoned(ctl)) drain_after_poison();
 }
 
 // ---- MMA issuer ----------------------------------------------------------------------------------
 __device__ void tc_mma_issuer(const TcParams& P, TcCtl* ctl, uint32_t smemA, uint32_t smemB, int cta, int G) {
     const TcArgs& a = P.a;
     const uint32_t tmem = ctl->tmem_base;
-    unsigned seg_cnt = 0, c_cnt = 0;
+    unsigned seg_cnt = 0, slot = 0, round = 0;
     for (int s = 0; s < a.k; ++s)
         for (int p = 0; p < PH_COUNT; ++p) {
             const PhaseShape sh = phase_shape(a, p);
-            long long idx = range_lo(sh.W, cta, G);
-            const long long hi = range_lo(sh.W, cta + 1, G);
-            while (idx < hi) {
-                const int kb0 = (int)(idx % sh.nkb);
-                const int n = (int)((hi - idx) < (long long)(sh.nkb - kb0) ? (hi - idx) : (long long)(sh.nkb - kb0));
+            const long long lo = range_lo(sh.W, cta, G), hi = range_lo(sh.W, cta + 1, G);
+            int left = (int)(hi - lo);
+            int kb0 = left > 0 ? (int)(lo % sh.nkb) : 0;
+            while (left > 0) {
+                const int n = left < sh.nkb - kb0 ? left : sh.nkb - kb0;
                 const unsigned acc = seg_cnt & 1u, use = seg_cnt >> 1;
                 if (use > 0) wait_mbar(saddr(&ctl->tempty[acc]), (use - 1) & 1u, ctl, a.error_flag, 4);
                 tc_fence_after();
                 for (int j = 0; j < n; ++j) {
-                    const unsigned slot = c_cnt % TC_STAGES;
-                    const bool ok = wait_mbar(saddr(&ctl->full[slot]), (c_cnt / TC_STAGES) & 1u, ctl, a.error_flag, 5);
+                    const bool ok = wait_mbar(saddr(&ctl->full[slot]), round & 1u, ctl, a.error_flag, 5);
                     if (ok) {
                         tc_fence_after();
                         const u64 ad = tc_smem_desc(smemA + slot * TC_A_BYTES);
@@ -378,11 +376,12 @@ __device__ void tc_mma_issuer(const TcParams& P, TcCtl* ctl, uint32_t smemA, uin
                             tc_mma(tmem + acc * TC_TN, ad + (u64)(kk * 2), bd + (u64)(kk * 2), (j > 0 || kk > 0) ? 1u : 0u);
                         tc_commit(saddr(&ctl->empty[slot]));
                     }
-                    ++c_cnt;
+                    if (++slot == TC_STAGES) { slot = 0; ++round; }
                 }
                 if (!poisoned(ctl)) tc_commit(saddr(&ctl->tfull[acc]));
                 ++seg_cnt;
-                idx += n;
+                left -= n;
+                kb0 = 0;
             }
         }
 }
@@ -612,16 +611,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
     tc_fence_after();
 
     if (warp == 0) {
-        if (lane == 0) tc_producer(P, ctl, smemA, smemB, cta, G);
+        if (lane == 0) tc_producer_w(P, ctl, smemA, cta, G);
         __syncwarp();
     } else if (warp == 1) {
         if (lane == 0) tc_mma_issuer(P, ctl, smemA, smemB, cta, G);
         __syncwarp();
-    } else {
-        // warps 2..7: attention; warps 4..7 also the epilogue of every GEMM phase
-        const int atid = tid - 64;
+    } else if (warp == 2) {
+        tc_producer_x(P, ctl, smemB, cta, G, lane);
+    } else if (warp >= 4) {
+        // warps 4..7: epilogue of every GEMM phase, and the attention between the QKV and O phases
+        const int etid = tid - 128;
         const int w4 = warp - 4;
-        const bool is_epi = warp >= 4;
         unsigned seg_cnt = 0;
         AttnArgs aa;
         aa.qkv = a.qkv; aa.ld = a.qw + 2 * a.kvw; aa.Kc = a.Kc; aa.Vc = a.Vc; aa.slots = a.slots; aa.pos0 = a.pos0;
@@ -632,35 +632,31 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
         const int hgroups = a.Hq / GQ;
         const int nunits = a.B * hgroups * a.attn_nsplit;
         for (int s = 0; s < a.k; ++s) {
-            if (is_epi) {
-                tc_epilogue_phase(P, ctl, s, PH_FC, seg_cnt, cta, G, w4, lane);
-                tc_epilogue_phase(P, ctl, s, PH_QKV, seg_cnt, cta, G, w4, lane);
-            }
+            tc_epilogue_phase(P, ctl, s, PH_FC, seg_cnt, cta, G, w4, lane);
+            tc_epilogue_phase(P, ctl, s, PH_QKV, seg_cnt, cta, G, w4, lane);
             // ---- attention: needs every CTA's QKV rows
-            if (atid == 0)
+            if (etid == 0)
                 wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(s * TC_BARS_PER_STEP + 2), ctl, a.error_flag, 7);
-            named_sync(TC_BAR_ATT, TC_ATT_THREADS);
+            named_sync(TC_BAR_EPI, TC_EPI_THREADS);
             if (!poisoned(ctl)) {
                 for (int unit = cta; unit < nunits; unit += G) {
                     const int split = unit % a.attn_nsplit;
                     const int rest = unit / a.attn_nsplit;
                     const int hg = rest % hgroups, b = rest / hgroups;
-                    attn_unit<bf16, DH, GQ, TC_ATT_WARPS, TC_BAR_ATT>(aa, split, hg, b, __ldg(a.pos0 + b) + s,
-                                                                      __ldg(a.slots + b), *asm_, atid);
+                    attn_unit<bf16, DH, GQ, TC_ATT_WARPS, TC_BAR_EPI>(aa, split, hg, b, __ldg(a.pos0 + b) + s,
+                                                                      __ldg(a.slots + b), *asm_, etid);
                 }
             }
             __threadfence();
-            named_sync(TC_BAR_ATT, TC_ATT_THREADS);
-            if (atid == 0) {
+            named_sync(TC_BAR_EPI, TC_EPI_THREADS);
+            if (etid == 0) {
                 fence_proxy_async_all();
                 red_release_add_u64(a.bar_counter, 1ull);
             }
-            if (is_epi) {
-                tc_epilogue_phase(P, ctl, s, PH_O, seg_cnt, cta, G, w4, lane);
-                tc_epilogue_phase(P, ctl, s, PH_GU, seg_cnt, cta, G, w4, lane);
-                tc_epilogue_phase(P, ctl, s, PH_DOWN, seg_cnt, cta, G, w4, lane);
-                tc_epilogue_phase(P, ctl, s, PH_LM, seg_cnt, cta, G, w4, lane);
-            }
+            tc_epilogue_phase(P, ctl, s, PH_O, seg_cnt, cta, G, w4, lane);
+            tc_epilogue_phase(P, ctl, s, PH_GU, seg_cnt, cta, G, w4, lane);
+            tc_epilogue_phase(P, ctl, s, PH_DOWN, seg_cnt, cta, G, w4, lane);
+            tc_epilogue_phase(P, ctl, s, PH_LM, seg_cnt, cta, G, w4, lane);
         }
     }
     tc_fence_before();
