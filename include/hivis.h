@@ -172,14 +172,15 @@ int hivis_read_kv(hivis_ctx* ctx, int slot, int row0, int n, float* out_k, float
 enum { HIVIS_TAP_U = 0, HIVIS_TAP_ATTN = 1, HIVIS_TAP_Y = 2, HIVIS_TAP_ACT = 3, HIVIS_TAP_G = 4 };
 int hivis_debug_tap(hivis_ctx* ctx, int which, float* out, void* stream);
 
-/* Options.  HIVIS_OPT_TC_KERNEL (default 1): with bf16 weights, d a multiple of 64 and at most 16
- * sequences, a draft runs all k steps in one persistent cooperative kernel that streams the weights
- * with TMA and multiplies on the tcgen05 tensor cores (weights as the M operand, batch as N); 0 falls
- * back to the kernels below.  HIVIS_OPT_CHAIN_KERNEL (default 1): a draft of ONE sequence runs all k steps in a
- * single persistent cooperative kernel (one CTA per SM, grid barriers between the phases of a step,
- * weights prefetched across them); 0 runs the same steps as separate kernel launches, which is what
- * batches of two or more sequences always use.  Both give the same results up to fp32 summation
- * order.                                                                                        */
+/* Options.
+ * HIVIS_OPT_CHAIN_KERNEL (default 1): a draft of ONE sequence runs all k steps in a single persistent
+ * cooperative kernel of fp32 FMAs (one CTA per SM, grid barriers between the phases of a step, weights
+ * prefetched across them by per-warp bulk-copy rings).
+ * HIVIS_OPT_TC_KERNEL (default 1): with bf16 weights and d a multiple of 64, a draft of 2..16 sequences
+ * runs all k steps in one persistent cooperative kernel that streams the weights with TMA and multiplies
+ * on the tcgen05 tensor cores (weights as the M operand, batch as N); 2 = use it for one sequence as well;
+ * 0 = never.  What neither kernel takes runs as separate kernel launches per step.  All paths give the
+ * same results up to fp32 summation order and the bf16 rounding of the tensor-core operand.            */
 enum { HIVIS_OPT_CHAIN_KERNEL = 0, HIVIS_OPT_TC_KERNEL = 1 };
 int hivis_set_option(hivis_ctx* ctx, int option, int value);
 

@@ -285,8 +285,10 @@ class Drafter:
     def set_chain_kernel(self, on: bool):
         hivis_set_option(self.ctx, HIVIS_OPT_CHAIN_KERNEL, 1 if on else 0)
 
-    def set_tc_kernel(self, on: bool):
-        hivis_set_option(self.ctx, HIVIS_OPT_TC_KERNEL, 1 if on else 0)
+    def set_tc_kernel(self, on):
+        """False/0: never; True: for every batch size it supports (2 in the C API); "auto"/1: the default."""
+        v = 1 if on == "auto" else (2 if on is True else int(on))
+        hivis_set_option(self.ctx, HIVIS_OPT_TC_KERNEL, v)
 
     def status(self):
         hivis_status(self.ctx)

@@ -12,7 +12,7 @@ OUT = os.path.join(HERE, "libhivis.so")
 OBJ_DIR = os.path.join(HERE, "_build")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-         "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall"]
+         "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall"] + os.environ.get("HIVIS_NVCC_FLAGS", "").split()
 
 
 def sources():

@@ -43,7 +43,7 @@ struct hivis_ctx {
     int* error_flag;
     // tensor-core chain kernel (bf16, up to 16 sequences)
     bool tc_ok;                   // cooperative launch available, shapes supported, tensor maps built
-    bool opt_tc;                  // option HIVIS_OPT_TC_KERNEL
+    int opt_tc;                   // option HIVIS_OPT_TC_KERNEL: 0 off, 1 for two or more sequences, 2 always
     TcMaps tc_maps;
     float* tc_partial;
     int* tile_ctr;
@@ -245,7 +245,7 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
     if (c->nsplit_cap > 64) c->nsplit_cap = 64;
     c->opt_chain = true;
     c->chain_ok = false;
-    c->opt_tc = true;
+    c->opt_tc = 1;
     c->tc_ok = false;
     c->tc_partial = nullptr;
     c->tile_ctr = nullptr;
@@ -564,7 +564,30 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
         rc = prepare_rho(c, resid, n_resid, st);
         if (rc) return rc;
     }
-    if (c->tc_ok && c->opt_tc && B <= 16) {
+    if (B == 1 && c->opt_chain && c->chain_ok && !(c->tc_ok && c->opt_tc == 2)) {
+        // one sequence: all k steps in one persistent cooperative kernel
+        ChainArgs a;
+        fill_chain_args(c, &a);
+        a.k = k;
+        a.rho = resid ? c->rho : nullptr;
+        a.n_resid = resid ? n_resid : 1;
+        a.slot = sl.slot[0];
+        a.forced = forced_ids;
+        a.logits_out = out_logits;
+        a.out_ids = out_ids;
+        plan_attention(c, max_rows, c->num_sms / g.n_q_heads, &a.attn_chunk, &a.attn_nsplit);
+        a.bar_base = c->bar_count_host;
+        CKP(c, CLS_CHAIN, st, launch_draft_chain(a, c->dtype, c->num_sms, st));
+        c->bar_count_host += (u64)c->num_sms * (u64)(chain_barriers_per_step() * k);
+        const int s0 = sl.slot[0];
+        c->kv_upper[s0] += k;
+        c->pending[s0] = false;
+        c->last_k[s0] = k;
+        c->tap_B = 1;
+        c->tap_mma = false;
+        return HIVIS_OK;
+    }
+    if (c->tc_ok && c->opt_tc != 0 && B <= 16) {
         // bf16, up to 16 sequences: all k steps in one cooperative tensor-core kernel
         const int lo = B <= 8 ? 1 : 0;
         CKP(c, CLS_OTHER, st, launch_tc_setup(sl, k, d, lo, c->d_slots, c->d_pos0, c->kv_len, c->pend_feat, c->pend_id,
@@ -604,29 +627,6 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
         }
         c->tap_B = B;
         c->tap_mma = true;
-        return HIVIS_OK;
-    }
-    if (B == 1 && c->opt_chain && c->chain_ok) {
-        // one sequence: all k steps in one persistent cooperative kernel
-        ChainArgs a;
-        fill_chain_args(c, &a);
-        a.k = k;
-        a.rho = resid ? c->rho : nullptr;
-        a.n_resid = resid ? n_resid : 1;
-        a.slot = sl.slot[0];
-        a.forced = forced_ids;
-        a.logits_out = out_logits;
-        a.out_ids = out_ids;
-        plan_attention(c, max_rows, c->num_sms / g.n_q_heads, &a.attn_chunk, &a.attn_nsplit);
-        a.bar_base = c->bar_count_host;
-        CKP(c, CLS_CHAIN, st, launch_draft_chain(a, c->dtype, c->num_sms, st));
-        c->bar_count_host += (u64)c->num_sms * (u64)(chain_barriers_per_step() * k);
-        const int s0 = sl.slot[0];
-        c->kv_upper[s0] += k;
-        c->pending[s0] = false;
-        c->last_k[s0] = k;
-        c->tap_B = 1;
-        c->tap_mma = false;
         return HIVIS_OK;
     }
     CKP(c, CLS_OTHER, st, launch_draft_setup(sl, k, d, c->d_slots, c->d_pos0, c->kv_len, c->pend_feat, c->pend_id, c->feat,
@@ -816,7 +816,8 @@ int hivis_set_option(hivis_ctx* c, int option, int value) {
         return HIVIS_OK;
     }
     if (option == HIVIS_OPT_TC_KERNEL) {
-        c->opt_tc = value != 0;
+        if (value < 0 || value > 2) return fail(c, HIVIS_ERR_ARG, "HIVIS_OPT_TC_KERNEL takes 0, 1 or 2");
+        c->opt_tc = value;
         return HIVIS_OK;
     }
     return fail(c, HIVIS_ERR_ARG, "unknown option %d", option);

@@ -1,6 +1,6 @@
 // Persistent draft-chain kernel for one sequence: all k chained draft steps in ONE cooperative launch.
 //
-// One CTA per SM, 8 warps.  Every weight matrix of the step (fusion FC, QKV, O, gate/up, down, LM
+// One CTA per SM, 16 warps.  Every weight matrix of the step (fusion FC, QKV, O, gate/up, down, LM
 // head) is split by rows across the CTAs; inside a CTA the rows are cut into chunks of at most 4 KB of
 // contiguous weights ("units") which the warps take round-robin.  Each warp owns a private ring of
 // shared-memory stages and keeps it full with bulk-async copies (cp.async.bulk + mbarrier
@@ -20,10 +20,16 @@
 // flag, waits (bounded) for its own copies in flight and returns.
 #include "attn_body.cuh"
 
-#define CHAIN_WARPS 8
+#ifndef CHAIN_WARPS
+#define CHAIN_WARPS 16
+#endif
 #define CHAIN_THREADS (CHAIN_WARPS * 32)
-#define CHAIN_STAGES 4
+#ifndef CHAIN_STAGES
+#define CHAIN_STAGES 2
+#endif
+#ifndef CHAIN_CHUNK_BYTES
 #define CHAIN_CHUNK_BYTES 4096
+#endif
 #define CHAIN_WAIT_CYCLES 2000000000ll      // ~1 s: far beyond any legitimate wait
 
 // ------------------------------------------------------------------------------------------ PTX helpers
