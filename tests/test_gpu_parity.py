@@ -329,3 +329,85 @@ def test_host_side_errors_do_not_launch():
         assert e.value.code == -4
     finally:
         case.close()
+
+
+# ---------------------------------------------------------------------------------------------------
+# Full-size workloads, in the launch configuration the benchmark times.  The CUDA path runs the whole
+# batch; the oracle (fp64, one sequence at a time) is run on sampled sequences: the shortest, the longest
+# and one more.  Every sampled sequence is compared completely: free-running ids (top-2-gap rule),
+# teacher-forced logits of every step, appended K/V rows and the verification outputs.
+# ---------------------------------------------------------------------------------------------------
+def _sampled_full_size(name, n_samples):
+    import torch
+    wl = hi.workload(name)
+    case = Case(wl)                       # builds the oracle object too; nothing is computed yet
+    try:
+        B, k = wl.batch, wl.k
+        lens = case.lens
+        order = np.argsort(lens, kind="stable")
+        picks = [int(order[0]), int(order[-1])] + [int(b) for b in order[1:-1][:: max(1, (B - 2) // max(1, n_samples - 2))]]
+        picks = sorted(set(picks))[:n_samples] if B > 1 else [0]
+        case.gpu_prefill()
+        ids_g, logits_g = case.gpu_draft(k)                               # free running, whole batch
+        rho = case.oracle.fold_residuals(case.resid)
+        refs = {}
+        for b in picks:
+            lo, hi_ = int(case.cu[b]), int(case.cu[b + 1])
+            T = hi_ - lo
+            Kc, Vc = case.oracle.new_cache(T + k)
+            case.oracle.prefill(case.ids[lo:hi_], case.hidden[lo:hi_], rho[0], Kc, Vc)
+            r = case.oracle.draft(T - 1, int(case.ids[hi_ - 1]), case.hidden[hi_ - 1], k, rho, Kc, Vc)
+            r["K"], r["V"], r["T"] = Kc, Vc, T
+            refs[b] = r
+            for s in range(k):
+                if ids_g[b, s] != r["ids"][s]:
+                    assert r["gaps"][s] < 1e-2, f"seq {b} step {s}: id {ids_g[b, s]} != {r['ids'][s]}, gap {r['gaps'][s]}"
+                    break
+                err = row_rel_err(logits_g[b, s], r["logits"][s])
+                assert err <= 2e-2, f"free run seq {b} step {s}: logits rel err {err}"
+        # teacher forcing: sampled sequences follow the oracle's ids, the others their own free-running ids
+        forced = ids_g.copy()
+        for b in picks:
+            forced[b] = refs[b]["ids"]
+        case.gpu_restore()
+        ids_f, logits_f = case.gpu_draft(k, forced=forced)
+        case.drafter.status()
+        for b in picks:
+            r = refs[b]
+            err = row_rel_err(logits_f[b], r["logits"])
+            assert err.max() <= 2e-2, f"teacher-forced seq {b}: logits rel err {err.max()}"
+            bad = (ids_f[b] != r["ids"]) & (r["gaps"] >= 1e-2)
+            assert not bad.any(), f"teacher-forced ids of seq {b} differ outside the gap zone"
+            n = r["T"] - 1 + k
+            k_g, v_g = case.drafter.read_kv(b, 0, n)
+            torch.cuda.synchronize()
+            for got, want in ((k_g, r["K"][:n]), (v_g, r["V"][:n])):
+                e = np.abs(got.cpu().numpy() - want).max() / np.abs(want).max()
+                assert e <= 1e-2, f"cache of seq {b}: rel err {e}"
+        # verification on the whole batch: planted accept lengths, sampled sequences against the oracle
+        logits_t, planted = hi.make_target_logits(wl, forced)
+        acc, nxt, kv = case.drafter.verify(torch.from_numpy(forced).cuda(), to_dev(logits_t, wl.logits_dtype))
+        torch.cuda.synchronize()
+        acc, nxt, kv = acc.cpu().numpy(), nxt.cpu().numpy(), kv.cpu().numpy()
+        np.testing.assert_array_equal(acc, planted)
+        for b in picks:
+            assert (int(acc[b]), int(nxt[b]), int(kv[b])) == case.oracle.verify(forced[b], logits_t[b], int(lens[b]))
+        # properties that hold for every sequence at any size
+        assert ((0 <= acc) & (acc <= k)).all()
+        np.testing.assert_array_equal(kv, lens + np.minimum(acc, k - 1))
+        np.testing.assert_array_equal(nxt, logits_t[np.arange(B), acc].argmax(-1))
+        assert ((0 <= ids_g) & (ids_g < wl.dims.vocab)).all()
+    finally:
+        case.close()
+
+
+def test_full_size_c2_llava_b1():
+    _sampled_full_size("c2_llava_b1", 1)
+
+
+def test_full_size_c3_llava_b16_ragged_sampled():
+    _sampled_full_size("c3_llava_b16_ragged", 3)
+
+
+def test_full_size_c4_qwen_b8_sampled():
+    _sampled_full_size("c4_qwen_b8", 2)
