@@ -53,7 +53,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE, text=True)
+                                          "-lms", "25", "-i", str(self.gpu)], stdout=subprocess.PIPE, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
         except Exception:
@@ -121,8 +121,8 @@ def run_oracle_sample(wl, steps: int, warmup: int):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2_llava_b1")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -265,6 +265,8 @@ def main():
         nbytes = k * step_bytes
         kern["draft_chain"] = {"us": round(us, 2), "launches_per_bench_step": 1,
                                "GBps": round(nbytes / (us * 1e-6) / 1e9, 1)}
+        kern["draft_chain"]["kernel"] = ("draft_chain_kernel (one sequence, fp32 FMA, all k steps in one launch)" if B == 1 else
+                                        "tc_chain_kernel (tcgen05, all k steps in one launch)")
         dom, dom_bytes = "draft_chain", nbytes
     else:
         dom = max((n for n in kern), key=lambda n: prof[n][0])
