@@ -242,7 +242,7 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
     const long long d = cfg->d, F = cfg->ffn, V = cfg->vocab, R = c->rows_cap, MB = cfg->max_batch;
     c->chunk = 128;
     c->nsplit_cap = (cfg->max_len + 31) / 32;
-    if (c->nsplit_cap > 64) c->nsplit_cap = 64;
+    if (c->nsplit_cap > 512) c->nsplit_cap = 512;
     c->opt_chain = true;
     c->chain_ok = false;
     c->opt_tc = 1;
@@ -351,7 +351,7 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
         fill_chain_args(c, &ca);
         c->chain_ok = chain_smem_bytes(ca, c->dtype, c->num_sms) != 0;
     }
-    if (c->dtype == HIVIS_BF16 && c->num_sms > 0 && c->chain_ok_coop &&
+    if (c->dtype == HIVIS_BF16 && c->num_sms > 0 && c->chain_ok_coop && (cfg->max_len + 31) / 32 <= c->nsplit_cap &&
         tc_supported(cfg->d, cfg->head_dim, cfg->n_q_heads, cfg->n_kv_heads, cfg->ffn)) {
         ChainArgs ca;
         fill_chain_args(c, &ca);
@@ -610,11 +610,7 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
         a.partial = c->tc_partial; a.tile_ctr = c->tile_ctr;
         a.Kc = c->Kc; a.Vc = c->Vc; a.inv_freq = c->inv_freq; a.part_acc = c->part_acc; a.part_ml = c->part_ml;
         a.counters = c->counters;
-        {
-            const int gq = (g.n_q_heads / g.n_kv_heads) % 7 == 0 ? 7 : 1;
-            const int groups = B * (g.n_q_heads / gq);
-            plan_attention(c, max_rows, (c->num_sms + groups - 1) / groups, &a.attn_chunk, &a.attn_nsplit);
-        }
+        a.attn_nslot = c->nsplit_cap;
         a.bar_counter = c->bar_counter; a.bar_base = c->bar_count_host; a.error_flag = c->error_flag;
         CKP(c, CLS_CHAIN, st, launch_tc_chain(c->tc_maps, a, c->num_sms, st));
         c->bar_count_host += (u64)c->num_sms * (u64)(tc_barriers_per_step() * k);

@@ -1,0 +1,372 @@
+// Warp-granular split-KV decode attention over the ragged text-only cache (bf16 cache), used by the
+// tensor-core chain kernel.
+//
+// Unit of work: 32 consecutive cache rows of one key = (sequence, group of GQ query heads on one KV head).  All units of the batch are laid out in (sequence, KV head, block) order and cut into equal
+// contiguous ranges, one per participating warp, whatever the sequence lengths: a ragged batch is balanced
+// to within one block.  No shared memory and no CTA-wide synchronisation is used.
+//
+// Inside a unit (DH = 128: a cache row is 16 lanes x 16 bytes, so one load instruction reads two whole rows):
+//   scores : every lane multiplies its 8-element slice of q with the matching slice of K for the rows it
+//            loaded; the slices are summed with a transposing butterfly (15 shuffles for 32 rows), after
+//            which each lane holds the complete score of ONE row;
+//   softmax: online (running max / sum) with warp shuffles;
+//   PV     : lane owns DH/32 output elements; V rows are read as whole rows (coalesced), the row's
+//            probability is broadcast from the lane that holds it.
+// A warp keeps accumulating while consecutive units belong to the same (sequence, KV head).  When the key
+// changes it writes the result - directly if it covered all blocks of the key, else as an unnormalised partial
+// (max, sum, acc) to global memory; the warp that completes the key's block count (arrival counter, nobody
+// waits) merges the partials in block order, so the result does not depend on arrival order.
+// The new position's K (rotated here) and V are appended to the cache by the unit that contains that row.
+#pragma once
+#include "attn_body.cuh"
+
+struct AttnWArgs {
+    const float* qkv;       // [B][ld] fp32: q | k | v of the new position, before RoPE
+    int ld;
+    bf16* Kc;               // [slot][Hkv][max_len][dh], K stored after RoPE
+    bf16* Vc;
+    const int* slots;       // [B]
+    const int* pos0;        // [B] cache row of draft step 0
+    int step;
+    const double* inv_freq; // [dh/2]
+    int Hq, Hkv, max_len, B;
+    float scale;
+    float* part_acc;        // [B][Hq][nslot][dh]
+    float* part_ml;         // [B][Hq][nslot][2]
+    int nslot;              // >= blocks of the longest sequence
+    int* counters;          // [B][Hq/GQ] blocks finished per key, zero between phases
+    float* attn;            // [B][Hq*dh] fp32
+    bf16* attn_h;           // [B][Hq*dh] bf16 (+ remainder rows when lo_rows > 0)
+    int lo_rows;
+};
+
+// Unit ranges of the warps.  32-bit arithmetic: units * warps stays far below 2^31 for every size the
+// library accepts (<= 16 sequences x 128 head groups x 512 blocks, a few thousand warps would still fit).
+__device__ __forceinline__ unsigned attw_lo(unsigned U, int g, int NW) { return U * (unsigned)g / (unsigned)NW; }
+__device__ __forceinline__ int attw_owner(unsigned U, int NW, unsigned u) {
+    int g = (int)(u * (unsigned)NW / U);
+    if (g >= NW) g = NW - 1;
+    while (g + 1 < NW && attw_lo(U, g + 1, NW) <= u) ++g;
+    while (g > 0 && attw_lo(U, g, NW) > u) --g;
+    return g;
+}
+
+// fp32 result and its bf16 operand copy (with the rounding remainder in row b + lo_rows when asked for)
+__device__ __forceinline__ void attw_store(const AttnWArgs& a, int b, int qw, int col, float o) {
+    a.attn[(long long)b * qw + col] = o;
+    const bf16 hi = __float2bfloat16_rn(o);
+    a.attn_h[(long long)b * qw + col] = hi;
+    if (a.lo_rows > 0) a.attn_h[(long long)(b + a.lo_rows) * qw + col] = __float2bfloat16_rn(o - __bfloat162float(hi));
+}
+
+// this lane's slice of a V row: DH/32 bf16 values in one load
+template <int EPL> struct AttwVec;
+template <> struct AttwVec<4> {
+    typedef uint2 type;
+    __device__ __forceinline__ static uint2 zero() { return make_uint2(0u, 0u); }
+    __device__ __forceinline__ static void unpack(uint2 w, float (&f)[4]) {
+        f[0] = bf16_lo(w.x); f[1] = bf16_hi(w.x); f[2] = bf16_lo(w.y); f[3] = bf16_hi(w.y);
+    }
+};
+template <> struct AttwVec<2> {
+    typedef unsigned type;
+    __device__ __forceinline__ static unsigned zero() { return 0u; }
+    __device__ __forceinline__ static void unpack(unsigned w, float (&f)[2]) { f[0] = bf16_lo(w); f[1] = bf16_hi(w); }
+};
+
+template <int DH, int GQ>
+__device__ void attn_warp_phase(const AttnWArgs& a, int gw, int NW, int lane) {
+    constexpr int LPR = DH / 8;          // lanes per cache row (16-byte slices)
+    constexpr int RPI = 32 / LPR;        // rows per load instruction
+    constexpr int NI = LPR;              // load instructions per 32-row block
+    constexpr int EPL = DH / 32;         // output elements per lane
+    constexpr int HALF = DH / 2;
+    const int c = lane % LPR, hrow = lane / LPR;
+    const int G = a.Hq / a.Hkv;
+    const int HG = a.Hq / GQ;            // keys per sequence
+    const int qw = a.Hq * DH, kvw = a.Hkv * DH;
+
+    // units of the batch
+    unsigned U = 0;
+    for (int b = 0; b < a.B; ++b) U += (unsigned)HG * (unsigned)((__ldg(a.pos0 + b) + a.step + 1 + 31) >> 5);
+    const unsigned u0 = attw_lo(U, gw, NW), u1 = attw_lo(U, gw + 1, NW);
+    if (u0 >= u1) return;
+
+    // locate the first unit
+    int b = 0;
+    unsigned cum = 0;            // first unit of sequence b
+    int len = 0, nb = 0;
+    for (;; ++b) {
+        len = __ldg(a.pos0 + b) + a.step + 1;
+        nb = (len + 31) >> 5;
+        if (u0 < cum + (unsigned)(HG * nb)) break;
+        cum += (unsigned)(HG * nb);
+    }
+    int hg = (int)((u0 - cum) / nb), j = (int)((u0 - cum) % nb);
+
+    float qf[GQ][8], cs8[8], sn8[8];
+    float m_run[GQ], l_run[GQ], acc[GQ][EPL];
+    bool fresh = true;           // state must be initialised for the current key
+    int j_first = 0, nblk = 0;   // first block and number of blocks of the running partial
+
+    for (unsigned u = u0; u < u1; ++u) {
+        const int p = len - 1;                       // the new position's row
+        const int slot = __ldg(a.slots + b);
+        const float* qkv = a.qkv + (long long)b * a.ld;
+        const int h0 = hg * GQ, kvh = h0 / G;
+        bf16* Kbase = a.Kc + ((long long)slot * a.Hkv + kvh) * (long long)a.max_len * DH;
+        bf16* Vbase = a.Vc + ((long long)slot * a.Hkv + kvh) * (long long)a.max_len * DH;
+        if (fresh) {
+            // rotation of this lane's slice [8c, 8c+8) at position p (the same for every head), then the slice
+            // of every query head of the group, rotated and scaled
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int d = 8 * c + e;
+                rope_cs(p, a.inv_freq[d < HALF ? d : d - HALF], cs8[e], sn8[e]);
+            }
+#pragma unroll
+            for (int g = 0; g < GQ; ++g) {
+                const float* q = qkv + (h0 + g) * DH;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int d = 8 * c + e;
+                    const float x = __ldcg(q + d), y = __ldcg(q + (d < HALF ? d + HALF : d - HALF));
+                    qf[g][e] = (d < HALF ? x * cs8[e] - y * sn8[e] : x * cs8[e] + y * sn8[e]) * a.scale;
+                }
+                m_run[g] = -INFINITY;
+                l_run[g] = 0.f;
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) acc[g][e] = 0.f;
+            }
+            j_first = j;
+            nblk = 0;
+            fresh = false;
+        }
+        const int base = j << 5;
+        const int r1 = min(len, base + 32);
+        const bool has_new = p >= base && p < r1;
+        // the new row: K rotated, rounded to what the cache will hold; V likewise
+        float knew[8];
+        if (has_new) {
+            const bool writer = (h0 % G) == 0 && hrow == 0;      // one key per KV head appends the row
+            const float* kx = qkv + qw + kvh * DH;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int d = 8 * c + e;
+                const float x = __ldcg(kx + d), y = __ldcg(kx + (d < HALF ? d + HALF : d - HALF));
+                const bf16 kb = __float2bfloat16_rn(d < HALF ? x * cs8[e] - y * sn8[e] : x * cs8[e] + y * sn8[e]);
+                knew[e] = __bfloat162float(kb);
+                if (writer) Kbase[(long long)p * DH + d] = kb;
+            }
+            if (writer) {
+                const float* vx = qkv + qw + kvw + kvh * DH;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) Vbase[(long long)p * DH + 8 * c + e] = __float2bfloat16_rn(__ldcg(vx + 8 * c + e));
+            }
+        }
+        // ---- all loads of the unit go out first: the K slices of this lane's rows and (for VPRE rows) this
+        //      lane's slice of the V rows, so that a unit costs one memory round trip, not one per group
+        constexpr int VPRE = GQ == 1 ? 32 : 16;      // V rows requested before the scores (registers permitting)
+        typedef typename AttwVec<EPL>::type vec_t;
+        const int nrows = r1 - base;
+        uint4 kw[NI];
+#pragma unroll
+        for (int t = 0; t < NI; ++t) {
+            const int row = base + t * RPI + hrow;
+            kw[t] = make_uint4(0, 0, 0, 0);
+            if (row < r1 && row != p) kw[t] = __ldcg((const uint4*)(Kbase + (long long)row * DH + 8 * c));
+        }
+        vec_t vw[VPRE];
+#pragma unroll
+        for (int t = 0; t < VPRE; ++t) {
+            vw[t] = AttwVec<EPL>::zero();
+            if (t < nrows && base + t != p) vw[t] = __ldcg((const vec_t*)(Vbase + (long long)(base + t) * DH + lane * EPL));
+        }
+        // the new row's V slice (what the cache will hold)
+        float vnew[EPL];
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) vnew[e] = 0.f;
+        if (has_new) {
+            const float* vx = qkv + qw + kvw + kvh * DH + lane * EPL;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) vnew[e] = __bfloat162float(__float2bfloat16_rn(__ldcg(vx + e)));
+        }
+        // ---- scores: partial dot products of this lane's slice, reduced eight load instructions at a time
+        float sc[GQ];            // the complete score of row (base + c*RPI + hrow), one per head
+#pragma unroll
+        for (int g = 0; g < GQ; ++g) sc[g] = 0.f;
+#pragma unroll
+        for (int i0 = 0; i0 < NI; i0 += 8) {
+#pragma unroll
+            for (int g = 0; g < GQ; ++g) {
+                float v[8];
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    const int row = base + (i0 + t) * RPI + hrow;
+                    float kf[8];
+                    if (row == p && has_new) {
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) kf[e] = knew[e];
+                    } else {
+                        const uint4 w = kw[i0 + t];
+                        kf[0] = bf16_lo(w.x); kf[1] = bf16_hi(w.x); kf[2] = bf16_lo(w.y); kf[3] = bf16_hi(w.y);
+                        kf[4] = bf16_lo(w.z); kf[5] = bf16_hi(w.z); kf[6] = bf16_lo(w.w); kf[7] = bf16_hi(w.w);
+                    }
+                    float s = 0.f;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) s = fmaf(qf[g][e], kf[e], s);
+                    v[t] = s;
+                }
+                // transposing butterfly over the lanes of a row: afterwards v[0] is the sum for t = c & 7
+#pragma unroll
+                for (int off = 4; off >= 1; off >>= 1) {
+                    const bool up = (c & off) != 0;
+#pragma unroll
+                    for (int t = 0; t < off; ++t) {
+                        const float send = up ? v[t] : v[t + off];
+                        const float keep = up ? v[t + off] : v[t];
+                        v[t] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+                    }
+                }
+                if (LPR == 16) {
+                    v[0] += __shfl_xor_sync(0xffffffffu, v[0], 8);      // the other eight lanes of the row
+                    if ((c >> 3) == (i0 >> 3)) sc[g] = v[0];            // this group of eight holds instruction c
+                } else {
+                    sc[g] = v[0];
+                }
+            }
+        }
+        const int myrow = base + c * RPI + hrow;
+        const bool ok = myrow < r1;
+        // ---- online softmax over the block
+        float pr[GQ];
+#pragma unroll
+        for (int g = 0; g < GQ; ++g) {
+            const float sv = ok ? sc[g] : -INFINITY;
+            float mb = sv;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, o));
+            const float mn = fmaxf(m_run[g], mb);           // finite: the block has at least one row
+            const float corr = expf(m_run[g] - mn);
+            pr[g] = ok ? expf(sv - mn) : 0.f;
+            float ps = pr[g];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, o);
+            l_run[g] = l_run[g] * corr + ps;
+            m_run[g] = mn;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) acc[g][e] *= corr;
+        }
+        // ---- PV: row r's probability sits in lane (r % RPI) * LPR + r / RPI
+#pragma unroll
+        for (int h0v = 0; h0v < 32; h0v += VPRE) {
+            if (h0v > 0) {
+                if (h0v >= nrows) break;
+#pragma unroll
+                for (int t = 0; t < VPRE; ++t) {
+                    vw[t] = AttwVec<EPL>::zero();
+                    if (h0v + t < nrows && base + h0v + t != p)
+                        vw[t] = __ldcg((const vec_t*)(Vbase + (long long)(base + h0v + t) * DH + lane * EPL));
+                }
+            }
+#pragma unroll
+            for (int t = 0; t < VPRE; ++t) {
+                const int r = h0v + t;
+                float vf[EPL];
+                AttwVec<EPL>::unpack(vw[t], vf);
+                if (has_new && base + r == p) {
+#pragma unroll
+                    for (int e = 0; e < EPL; ++e) vf[e] = vnew[e];
+                }
+                const int src = (r % RPI) * LPR + r / RPI;
+#pragma unroll
+                for (int g = 0; g < GQ; ++g) {
+                    const float pj = __shfl_sync(0xffffffffu, pr[g], src);          // 0 for rows beyond the block
+#pragma unroll
+                    for (int e = 0; e < EPL; ++e) acc[g][e] = fmaf(pj, vf[e], acc[g][e]);
+                }
+            }
+        }
+        ++nblk;
+
+        // ---- next unit; flush when the key changes or this warp's range ends
+        const int b_cur = b, hg_cur = hg, nb_cur = nb;
+        const unsigned k0 = cum + (unsigned)(hg * nb);               // first unit of the current key
+        bool key_ends = false;
+        if (++j == nb) {
+            j = 0;
+            key_ends = true;
+            if (++hg == HG) {
+                hg = 0;
+                cum += (unsigned)(HG * nb);
+                ++b;
+                if (b < a.B) {
+                    len = __ldg(a.pos0 + b) + a.step + 1;
+                    nb = (len + 31) >> 5;
+                }
+            }
+        }
+        if (!key_ends && u + 1 < u1) continue;
+        fresh = true;
+        if (nblk == nb_cur) {
+            // the whole key was done here: write the result
+#pragma unroll
+            for (int g = 0; g < GQ; ++g)
+#pragma unroll
+                for (int e = 0; e < EPL; ++e)
+                    attw_store(a, b_cur, qw, (hg_cur * GQ + g) * DH + lane * EPL + e, acc[g][e] / l_run[g]);
+            continue;
+        }
+        // publish the partial in the slot of its first block
+#pragma unroll
+        for (int g = 0; g < GQ; ++g) {
+            const long long pi = ((long long)b_cur * a.Hq + hg_cur * GQ + g) * a.nslot + j_first;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) __stcg(a.part_acc + pi * DH + lane * EPL + e, acc[g][e]);
+            if (lane == 0) {
+                __stcg(a.part_ml + pi * 2, m_run[g]);
+                __stcg(a.part_ml + pi * 2 + 1, l_run[g]);
+            }
+        }
+        __threadfence();
+        __syncwarp();
+        int last = 0;
+        if (lane == 0) {
+            int* ctr = a.counters + b_cur * HG + hg_cur;
+            const int old = atomicAdd(ctr, nblk);
+            last = (old + nblk == nb_cur);
+            if (last) *ctr = 0;
+        }
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (!last) continue;
+        __threadfence();
+        // merge the key's partials in block order (a partial starts where a warp's range meets the key), one
+        // pass with running rescaling, all heads of the group per partial
+        float M[GQ], L[GQ], A[GQ][EPL];
+#pragma unroll
+        for (int g = 0; g < GQ; ++g) {
+            M[g] = -INFINITY;
+            L[g] = 0.f;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) A[g][e] = 0.f;
+        }
+        for (unsigned uu = k0; uu < k0 + (unsigned)nb_cur;) {
+#pragma unroll
+            for (int g = 0; g < GQ; ++g) {
+                const long long pi = ((long long)b_cur * a.Hq + hg_cur * GQ + g) * a.nslot + (uu - k0);
+                const float m = __ldcg(a.part_ml + pi * 2), l = __ldcg(a.part_ml + pi * 2 + 1);
+                const float Mn = fmaxf(M[g], m);
+                const float fo = expf(M[g] - Mn), fn = expf(m - Mn);
+                L[g] = L[g] * fo + l * fn;
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) A[g][e] = A[g][e] * fo + __ldcg(a.part_acc + pi * DH + lane * EPL + e) * fn;
+                M[g] = Mn;
+            }
+            uu = attw_lo(U, attw_owner(U, NW, uu) + 1, NW);
+        }
+#pragma unroll
+        for (int g = 0; g < GQ; ++g)
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) attw_store(a, b_cur, qw, (hg_cur * GQ + g) * DH + lane * EPL + e, A[g][e] / L[g]);
+    }
+}

@@ -172,7 +172,7 @@ struct TcArgs {
     const double* inv_freq;
     float *part_acc, *part_ml;
     int* counters;
-    int attn_chunk, attn_nsplit;
+    int attn_nslot;            // partial slots per (sequence, head): >= 32-row blocks of the longest sequence
     u64* bar_counter;
     u64 bar_base;
     int* error_flag;

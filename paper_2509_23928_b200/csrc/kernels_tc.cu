@@ -33,10 +33,10 @@
 // barriers still pair up, tensor memory is freed and the kernel returns.
 #include <cuda.h>
 
-#include "attn_body.cuh"
+#include "attn_warp.cuh"
 
 #define TC_THREADS 256
-#define TC_STAGES 10
+#define TC_STAGES 11
 #define TC_BK 64
 #define TC_TM 128
 #define TC_TN 16
@@ -583,8 +583,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
     const uint32_t smemA = saddr(smem);
     const uint32_t smemB = smemA + TC_STAGES * TC_A_BYTES;
     TcCtl* ctl = (TcCtl*)(smem + TC_STAGES * (TC_A_BYTES + TC_B_BYTES));
-    typedef AttnSmem<TC_ATT_WARPS, GQ, DH> ASm;
-    ASm* asm_ = (ASm*)(smem + TC_STAGES * (TC_A_BYTES + TC_B_BYTES) + ((sizeof(TcCtl) + 127) & ~(size_t)127));
 
     if (tid == 0) {
         for (int i = 0; i < TC_STAGES; ++i) {
@@ -623,14 +621,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
         const int etid = tid - 128;
         const int w4 = warp - 4;
         unsigned seg_cnt = 0;
-        AttnArgs aa;
-        aa.qkv = a.qkv; aa.ld = a.qw + 2 * a.kvw; aa.Kc = a.Kc; aa.Vc = a.Vc; aa.slots = a.slots; aa.pos0 = a.pos0;
-        aa.step = 0; aa.inv_freq = a.inv_freq; aa.Hq = a.Hq; aa.Hkv = a.Hkv; aa.dh = a.dh; aa.max_len = a.max_len;
-        aa.B = a.B; aa.scale = a.scale; aa.chunk = a.attn_chunk; aa.nsplit = a.attn_nsplit; aa.part_acc = a.part_acc;
-        aa.part_ml = a.part_ml; aa.counters = a.counters; aa.attn = a.attn; aa.attn_h = a.attn_h;
-        aa.lo_rows = a.lo ? a.B : 0;
-        const int hgroups = a.Hq / GQ;
-        const int nunits = a.B * hgroups * a.attn_nsplit;
+        AttnWArgs aw;
+        aw.qkv = a.qkv; aw.ld = a.qw + 2 * a.kvw; aw.Kc = (bf16*)a.Kc; aw.Vc = (bf16*)a.Vc; aw.slots = a.slots;
+        aw.pos0 = a.pos0; aw.step = 0; aw.inv_freq = a.inv_freq; aw.Hq = a.Hq; aw.Hkv = a.Hkv; aw.max_len = a.max_len;
+        aw.B = a.B; aw.scale = a.scale; aw.part_acc = a.part_acc; aw.part_ml = a.part_ml; aw.nslot = a.attn_nslot;
+        aw.counters = a.counters; aw.attn = a.attn; aw.attn_h = a.attn_h; aw.lo_rows = a.lo ? a.B : 0;
         for (int s = 0; s < a.k; ++s) {
             tc_epilogue_phase(P, ctl, s, PH_FC, seg_cnt, cta, G, w4, lane);
             tc_epilogue_phase(P, ctl, s, PH_QKV, seg_cnt, cta, G, w4, lane);
@@ -639,13 +634,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
                 wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(s * TC_BARS_PER_STEP + 2), ctl, a.error_flag, 7);
             named_sync(TC_BAR_EPI, TC_EPI_THREADS);
             if (!poisoned(ctl)) {
-                for (int unit = cta; unit < nunits; unit += G) {
-                    const int split = unit % a.attn_nsplit;
-                    const int rest = unit / a.attn_nsplit;
-                    const int hg = rest % hgroups, b = rest / hgroups;
-                    attn_unit<bf16, DH, GQ, TC_ATT_WARPS, TC_BAR_EPI>(aa, split, hg, b, __ldg(a.pos0 + b) + s,
-                                                                      __ldg(a.slots + b), *asm_, etid);
-                }
+                aw.step = s;
+                attn_warp_phase<DH, GQ>(aw, cta * TC_ATT_WARPS + w4, G * TC_ATT_WARPS, lane);
             }
             __threadfence();
             named_sync(TC_BAR_EPI, TC_EPI_THREADS);
@@ -770,8 +760,7 @@ cudaError_t tc_build_maps(TcMaps* maps, const ChainPhase* ph, int d, int qw, int
 template <int DH, int GQ>
 static cudaError_t tc_launch_t(const TcParams& P, int grid, cudaStream_t st) {
     static bool attr_set = false;
-    const size_t smem = 1024 + (size_t)TC_STAGES * (TC_A_BYTES + TC_B_BYTES) + ((sizeof(TcCtl) + 127) & ~(size_t)127) +
-                        sizeof(AttnSmem<TC_ATT_WARPS, GQ, DH>);
+    const size_t smem = 1024 + (size_t)TC_STAGES * (TC_A_BYTES + TC_B_BYTES) + ((sizeof(TcCtl) + 127) & ~(size_t)127);
     if (smem > 227 * 1024) return cudaErrorInvalidValue;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(tc_chain_kernel<DH, GQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
