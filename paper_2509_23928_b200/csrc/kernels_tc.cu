@@ -62,7 +62,7 @@ struct TcCtl {
     u64 full[TC_STAGES], empty[TC_STAGES], tfull[2], tempty[2];
     uint32_t tmem_base;
     int abort_flag;
-    int last_flag;
+    int last_flag, c_first, c_first_slot, n_contrib;
     float scale[16];
     float red[8][16];
 };
@@ -521,35 +521,72 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
         }
         bool finish = true;
         if (!(kb0 == 0 && n == sh.nkb)) {
-            // a tile shared with other CTAs: publish the partial accumulator; the last arriver finishes the tile
-            float* mine = a.partial + (long long)(cta * 2 + (idx == lo ? 0 : 1)) * (16 * TC_TM);
+            // a tile shared with other CTAs: publish the partial accumulator ([row][16 columns], 64 bytes per
+            // thread); the last arriver finishes the tile
+            float4* mine = (float4*)(a.partial + (long long)(cta * 2 + (idx == lo ? 0 : 1)) * (16 * TC_TM)) + etid * 4;
 #pragma unroll
-            for (int c = 0; c < 16; ++c) mine[c * TC_TM + etid] = v[c];
-            __threadfence();
+            for (int q = 0; q < 4; ++q) __stcg(mine + q, make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]));
             named_sync(TC_BAR_EPI, TC_EPI_THREADS);
             if (etid == 0) {
-                // contributors = the CTAs whose (non-empty) ranges meet this tile, in range order
+                // contributors = the CTAs whose (non-empty) ranges meet this tile, in range order; when every
+                // CTA has work in the phase they are consecutive CTAs
                 const long long t0 = (long long)tile * sh.nkb;
-                int nc = 0;
-                for (long long i = t0; i < t0 + sh.nkb; ++nc) i = range_lo(sh.W, owner_of(sh.W, G, i) + 1, G);
+                const int cf = owner_of(sh.W, G, t0);
+                int nc;
+                if (sh.W >= G) {
+                    nc = owner_of(sh.W, G, t0 + sh.nkb - 1) - cf + 1;
+                } else {
+                    nc = 0;
+                    for (long long i = t0; i < t0 + sh.nkb; ++nc) i = range_lo(sh.W, owner_of(sh.W, G, i) + 1, G);
+                }
+                ctl->c_first = cf;
+                ctl->c_first_slot = t0 == range_lo(sh.W, cf, G) ? 0 : 1;
+                ctl->n_contrib = nc;
+                __threadfence();                       // the CTA's partial (ordered before by the barrier) is visible first
                 const int old = atomicAdd(a.tile_ctr + tile, 1);
                 const int last = old == nc - 1;
-                if (last) a.tile_ctr[tile] = 0;
+                if (last) {
+                    a.tile_ctr[tile] = 0;
+                    __threadfence();
+                }
                 ctl->last_flag = last;
             }
             named_sync(TC_BAR_EPI, TC_EPI_THREADS);
             finish = ctl->last_flag != 0;
             if (finish) {
-                __threadfence();
-                const long long t0 = (long long)tile * sh.nkb;
+                // contributor order is fixed, so the sum does not depend on who arrived last
 #pragma unroll
                 for (int c = 0; c < 16; ++c) v[c] = 0.f;
-                for (long long i = t0; i < t0 + sh.nkb;) {
-                    const int cc = owner_of(sh.W, G, i);
-                    const float* src = a.partial + (long long)(cc * 2 + (i == range_lo(sh.W, cc, G) ? 0 : 1)) * (16 * TC_TM);
+                if (sh.W >= G) {
+                    const int cf = ctl->c_first, nc = ctl->n_contrib, fs = ctl->c_first_slot;
+                    const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 1
+                    for (int j0 = 0; j0 < nc; j0 += 2) {        // loads of two contributors in flight together
+                        const float4* sa = (const float4*)(a.partial + (long long)((cf + j0) * 2 + (j0 == 0 ? fs : 0)) * (16 * TC_TM)) + etid * 4;
+                        const float4* sb = (const float4*)(a.partial + (long long)((cf + j0 + 1) * 2) * (16 * TC_TM)) + etid * 4;
+                        const bool two = j0 + 1 < nc;
+                        const float4 a0 = __ldcg(sa), a1 = __ldcg(sa + 1), a2 = __ldcg(sa + 2), a3 = __ldcg(sa + 3);
+                        const float4 b0 = two ? __ldcg(sb) : z4, b1 = two ? __ldcg(sb + 1) : z4;
+                        const float4 b2 = two ? __ldcg(sb + 2) : z4, b3 = two ? __ldcg(sb + 3) : z4;
+                        v[0] += a0.x; v[1] += a0.y; v[2] += a0.z; v[3] += a0.w; v[4] += a1.x; v[5] += a1.y; v[6] += a1.z; v[7] += a1.w;
+                        v[8] += a2.x; v[9] += a2.y; v[10] += a2.z; v[11] += a2.w; v[12] += a3.x; v[13] += a3.y; v[14] += a3.z; v[15] += a3.w;
+                        if (two) {
+                            v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+                            v[8] += b2.x; v[9] += b2.y; v[10] += b2.z; v[11] += b2.w; v[12] += b3.x; v[13] += b3.y; v[14] += b3.z; v[15] += b3.w;
+                        }
+                    }
+                } else {
+                    const long long t0 = (long long)tile * sh.nkb;
+                    for (long long i = t0; i < t0 + sh.nkb;) {
+                        const int cc = owner_of(sh.W, G, i);
+                        const float4* src = (const float4*)(a.partial + (long long)(cc * 2 + (i == range_lo(sh.W, cc, G) ? 0 : 1)) * (16 * TC_TM)) + etid * 4;
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) v[c] += __ldcg(src + c * TC_TM + etid);
-                    i = range_lo(sh.W, cc + 1, G);
+                        for (int q = 0; q < 4; ++q) {
+                            const float4 t = __ldcg(src + q);
+                            v[4 * q] += t.x; v[4 * q + 1] += t.y; v[4 * q + 2] += t.z; v[4 * q + 3] += t.w;
+                        }
+                        i = range_lo(sh.W, cc + 1, G);
+                    }
                 }
             }
             named_sync(TC_BAR_EPI, TC_EPI_THREADS);      // last_flag may be rewritten by the next segment
@@ -560,7 +597,6 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
     // This CTA's part of the phase is done: arrive on the grid barrier.  All arrivals are counted in one
     // counter, so a CTA may arrive for this phase only once the barrier before it is complete.  With work in
     // the phase that is implied (its operand tiles were loaded after that barrier); without work, wait for it.
-    __threadfence();
     named_sync(TC_BAR_EPI, TC_EPI_THREADS);
     if (etid == 0) {
         const int need = need_seq(s, p);
