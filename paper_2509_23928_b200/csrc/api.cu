@@ -48,7 +48,7 @@ struct hivis_ctx {
     float* tc_partial;
     int* tile_ctr;
     int tc_tiles;
-    bf16* zero_row;
+    bf16* xe_h;
     int *slot_of, *row_of;
     long long map_cap;
     // host mirrors
@@ -288,7 +288,7 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
          dalloc(c, &c->part_ml, R * cfg->n_q_heads * (long long)c->nsplit_cap * 2) &&
          dalloc(c, &c->counters, R * cfg->n_q_heads) && dalloc(c, &c->bar_counter, 1) &&
          dalloc(c, &c->error_flag, 1) && dalloc(c, &c->slot_of, c->map_cap) &&
-         dalloc(c, &c->row_of, c->map_cap) && dalloc(c, &c->zero_row, d);
+         dalloc(c, &c->row_of, c->map_cap) && dalloc(c, &c->xe_h, R * d);
     if (!ok) {
         free_all(c);
         delete c;
@@ -329,7 +329,7 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
         CK(c, cudaMemsetAsync(c->counters, 0, R * cfg->n_q_heads * sizeof(int), st));
         CK(c, cudaMemsetAsync(c->bar_counter, 0, sizeof(u64), st));
         CK(c, cudaMemsetAsync(c->error_flag, 0, sizeof(int), st));
-        CK(c, cudaMemsetAsync(c->zero_row, 0, d * sizeof(bf16), st));
+        CK(c, cudaMemsetAsync(c->xe_h, 0, R * d * sizeof(bf16), st));
         CK(c, cudaMemsetAsync(c->feat_h, 0, R * d * sizeof(bf16), st));
         CK(c, cudaMemsetAsync(c->xq, 0, R * d * sizeof(bf16), st));
         CK(c, cudaMemsetAsync(c->attn_h, 0, R * c->qw * sizeof(bf16), st));
@@ -359,8 +359,8 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
         bool ok2 = dalloc(c, &c->tc_partial, (size_t)c->num_sms * 2 * 16 * 128) && dalloc(c, &c->tile_ctr, c->tc_tiles);
         if (ok2) ok2 = cudaMemsetAsync(c->tile_ctr, 0, c->tc_tiles * sizeof(int), st) == cudaSuccess;
         if (ok2)
-            ok2 = tc_build_maps(&c->tc_maps, ca.ph, cfg->d, c->qw, cfg->ffn, cfg->vocab, c->embed, c->feat_h, c->xq,
-                                c->attn_h, c->xm, c->act_h, c->zero_row) == cudaSuccess;
+            ok2 = tc_build_maps(&c->tc_maps, ca.ph, cfg->d, c->qw, cfg->ffn, c->feat_h, c->xq, c->attn_h, c->xm, c->act_h,
+                                c->xe_h) == cudaSuccess;
         if (!ok2) cudaGetLastError();
         c->tc_ok = ok2;
     }
@@ -591,7 +591,8 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
         // bf16, up to 16 sequences: all k steps in one cooperative tensor-core kernel
         const int lo = B <= 8 ? 1 : 0;
         CKP(c, CLS_OTHER, st, launch_tc_setup(sl, k, d, lo, c->d_slots, c->d_pos0, c->kv_len, c->pend_feat, c->pend_id,
-                                              c->feat, c->feat_h, c->cur_id, c->keys, c->key_stride, st));
+                                              c->feat, c->feat_h, c->cur_id, c->keys, c->key_stride, (const bf16*)c->embed,
+                                              V, c->xe_h, st));
         ChainArgs ca;
         fill_chain_args(c, &ca);
         TcArgs a;
@@ -606,6 +607,7 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
         a.keys = c->keys; a.key_stride = c->key_stride;
         a.u = c->u; a.qkv = c->qkv; a.attn = c->attn; a.y = c->y; a.feat = c->feat;
         a.feat_h = c->feat_h; a.xq_h = c->xq; a.attn_h = c->attn_h; a.xm_h = c->xm; a.act_h = c->act_h;
+        a.xe_h = c->xe_h; a.embed = (const bf16*)c->embed;
         a.ssq1 = c->ssq1; a.ssq2 = c->ssq2; a.logits_out = out_logits;
         a.partial = c->tc_partial; a.tile_ctr = c->tile_ctr;
         a.Kc = c->Kc; a.Vc = c->Vc; a.inv_freq = c->inv_freq; a.part_acc = c->part_acc; a.part_ml = c->part_ml;

@@ -143,8 +143,7 @@ struct CuSeqlens {
 #define TC_OP_ROWS 16          // rows of every bf16 operand buffer that the tensor maps cover
 enum { TCM_W = 0,              // PH_COUNT weight maps, box 64 x 128
        TCM_X_FEAT = PH_COUNT, TCM_X_XQ, TCM_X_ATTN, TCM_X_XM, TCM_X_ACT,   // operand maps, box 64 x 16
-       TCM_EMBED,              // embedding table, box 64 x 1 (one row per copy)
-       TCM_ZERO,               // one row of zeros, box 64 x 1
+       TCM_X_EMB,              // gathered embedding rows, box 64 x 16
        TCM_COUNT };
 struct TcMaps {
     alignas(64) unsigned char m[TCM_COUNT][128];     // CUtensorMap objects
@@ -164,6 +163,8 @@ struct TcArgs {
     int key_stride;
     float *u, *qkv, *attn, *y, *feat;     // fp32 activations [B][width]
     bf16 *feat_h, *xq_h, *attn_h, *xm_h, *act_h;   // bf16 operands [TC_OP_ROWS][width]
+    bf16* xe_h;                // [TC_OP_ROWS][d] embedding rows of the step's tokens (rows >= B stay zero)
+    const bf16* embed;         // [V][d]
     float *ssq1, *ssq2;        // [tiles*4][16] partial sums of squares of u / y
     float* logits_out;         // [B][k][V], nullable
     float* partial;            // [grid*2][16][128] split-tile partial accumulators
@@ -178,15 +179,15 @@ struct TcArgs {
     int* error_flag;
 };
 // fills `maps` for the given buffers; returns cudaSuccess or an error (driver entry point missing, bad shape)
-cudaError_t tc_build_maps(TcMaps* maps, const ChainPhase* ph, int d, int qw, int F, int V, const void* embed,
-                          const bf16* feat_h, const bf16* xq_h, const bf16* attn_h, const bf16* xm_h,
-                          const bf16* act_h, const bf16* zero_row);
+cudaError_t tc_build_maps(TcMaps* maps, const ChainPhase* ph, int d, int qw, int F, const bf16* feat_h,
+                          const bf16* xq_h, const bf16* attn_h, const bf16* xm_h, const bf16* act_h, const bf16* xe_h);
 bool tc_supported(int d, int dh, int Hq, int Hkv, int F);
 int tc_max_tiles(const ChainPhase* ph);
 cudaError_t launch_tc_chain(const TcMaps& maps, const TcArgs& a, int grid, cudaStream_t st);
 cudaError_t launch_tc_setup(const SlotList& sl, int k, int d, int lo, int* d_slots, int* d_pos0, int* kv_len,
                             const float* pend_feat, const int* pend_id, float* feat, bf16* feat_h,
-                            int* cur_id, u64* keys, int key_stride, cudaStream_t st);
+                            int* cur_id, u64* keys, int key_stride, const bf16* embed, int vocab, bf16* xe_h,
+                            cudaStream_t st);
 int tc_barriers_per_step();
 
 // ---------------------------------------------------------------------------------------------

@@ -6,16 +6,17 @@
 //                        ring with TMA (cp.async.bulk.tensor, 128-byte swizzle, mbarrier complete_tx).
 //                        Weight tiles do not depend on activations, so their loads run ahead through phase
 //                        and step boundaries, limited only by the ring.
-//   warp 2               operand producer: the matching batch-operand tiles (16 rows x 64 k, 2 KB) in the
+//   warp 2 (one thread)  operand producer: the matching batch-operand tiles (16 rows x 64 k, 2 KB) in the
 //                        same order; the first tile of a phase waits for the grid barrier before it.
+//   warp 3               embedding gather: once a step's tokens are known, copies their embedding rows into
+//                        the dense operand buffer of the fusion FC's embedding half (a barrier of its own).
 //   warp 1 (one thread)  issues tcgen05.mma (M = 128 weight rows, N = 16 batch columns, K = 16, four per
 //                        stage), accumulating in tensor memory (two 16-column accumulators, so the next
 //                        tile's MMAs overlap the previous tile's epilogue); tcgen05.commit frees stages.
 //   warps 4-7            epilogue: tcgen05.ld (one weight row per thread, 16 batch values), then the fused
 //                        output stage of the phase (residuals, RMSNorm statistics and gains, RoPE-free
 //                        QKV bias, SiLU*up, LM-head argmax keys) and the bf16 operand of the next phase.
-//                        Between the QKV and O phases the same warps run the split-KV attention over the
-//                        text-only cache.
+//   warps 3-7            between the QKV and O phases: split-KV attention over the text-only cache.
 //
 // Work split: a phase with T row tiles and KB k-blocks is T*KB tile-k-blocks, laid out tile-major and cut
 // into equal contiguous ranges, one per CTA (so every SM streams the same number of bytes whatever the
@@ -42,7 +43,8 @@
 #define TC_TN 16
 #define TC_A_BYTES (TC_TM * TC_BK * 2)
 #define TC_B_BYTES (TC_TN * TC_BK * 2)
-#define TC_ATT_WARPS 4               // the epilogue warps also run the attention
+#define TC_ATT_WARPS 5               // warps 3..7 run the attention
+#define TC_BAR_ATT 2
 #define TC_EPI_THREADS 128
 #define TC_BAR_EPI 3
 #define TC_WAIT_CYCLES 2000000000ll      // ~1 s: far beyond any legitimate wait
@@ -197,12 +199,14 @@ __device__ __forceinline__ bool wait_grid(const u64* counter, u64 target, TcCtl*
 }
 
 // ---- schedule --------------------------------------------------------------------------------------
-// grid barriers of one step, in order: after FC, QKV, attention, O, gate/up, down, LM head
-#define TC_BARS_PER_STEP 7
+// grid barriers of one step, in order: after the embedding gather, FC, QKV, attention, O, gate/up, down, LM head
+#define TC_BARS_PER_STEP 8
+#define TC_SEQ_GATHER 0
+#define TC_SEQ_ATTN 3
+__device__ __forceinline__ int phase_seq(int p) { return p < 2 ? p + 1 : p + 2; }       // barrier a GEMM phase arrives on
 __device__ __forceinline__ int need_seq(int step, int p) {                              // barrier its operand needs (-1: none)
-    if (p == PH_FC) return step == 0 ? -1 : (step - 1) * TC_BARS_PER_STEP + 6;
-    if (p == PH_QKV) return step * TC_BARS_PER_STEP + 0;
-    return step * TC_BARS_PER_STEP + p;              // O needs attention (2), GU needs O (3), DOWN 4, LM 5
+    if (p == PH_FC) return step == 0 ? -1 : (step - 1) * TC_BARS_PER_STEP + 7;       // hidden half: the previous LM head
+    return step * TC_BARS_PER_STEP + phase_seq(p) - 1;       // QKV needs FC, O needs attention, GU needs O, ...
 }
 struct PhaseShape {
     int nkb, ntiles;
@@ -282,15 +286,11 @@ __device__ void tc_producer_w(const TcParams& P, TcCtl* ctl, uint32_t smemA, int
     Cursor c{0, 0, 0, 0, 0, 0, true, false};
     cursor_enter(c, a, cta, G);
     unsigned slot = 0, round = 0;
-    const int dkb = a.d / TC_BK;
-    const int erows = a.lo ? 2 * a.B : a.B;
     while (c.live) {
         if (round > 0 && !wait_mbar(saddr(&ctl->empty[slot]), (round - 1) & 1u, ctl, a.error_flag, 3)) break;
         if (poisoned(ctl)) break;
         const uint32_t bar = saddr(&ctl->full[slot]);
-        // the embedding half of the fusion FC brings only the operand rows in use (one 128-byte row per copy)
-        const uint32_t xbytes = (c.p == PH_FC && c.kb >= dkb) ? (uint32_t)erows * 128u : (uint32_t)TC_B_BYTES;
-        mbar_expect_tx(bar, TC_A_BYTES + xbytes);
+        mbar_expect_tx(bar, TC_A_BYTES + TC_B_BYTES);
         tma_load_2d(smemA + slot * TC_A_BYTES, &P.maps.m[TCM_W + c.p], c.kb * TC_BK, c.tile * TC_TM, bar, pol_w);
         cursor_next(c, a, cta, G);
         if (++slot == TC_STAGES) { slot = 0; ++round; }
@@ -298,19 +298,18 @@ __device__ void tc_producer_w(const TcParams& P, TcCtl* ctl, uint32_t smemA, int
     if (poisoned(ctl)) drain_after_poison();
 }
 
-// Batch-operand tiles: same k-block order; the first tile of a phase waits for the grid barrier after
-// which the operand is complete.  Run by a whole warp with uniform control flow: lane 0 issues the tile
-// copies, and in the embedding half of the fusion FC lane r issues the copy of operand row r.
-__device__ void tc_producer_x(const TcParams& P, TcCtl* ctl, uint32_t smemB, int cta, int G, int lane) {
+// Batch-operand tiles (one thread): same k-block order; the first tile of a phase waits for the grid barrier
+// after which the operand is complete.  The embedding half of the fusion FC reads the rows that the gather
+// of this step copied out of the embedding table, and waits for that barrier.
+__device__ void tc_producer_x(const TcParams& P, TcCtl* ctl, uint32_t smemB, int cta, int G) {
     const TcArgs& a = P.a;
     const u64 pol_x = policy_evict_last();
     Cursor c{0, 0, 0, 0, 0, 0, true, false};
     cursor_enter(c, a, cta, G);
     unsigned slot = 0, round = 0;
-    int my_id = 0;
     const int dkb = a.d / TC_BK;
-    const int erows = a.lo ? 2 * a.B : a.B;
     int map_idx = TCM_X_FEAT;
+    int gathered_step = -1;
     while (c.live) {
         if (c.entered) {
             const int need = need_seq(c.step, c.p);
@@ -319,34 +318,58 @@ __device__ void tc_producer_x(const TcParams& P, TcCtl* ctl, uint32_t smemB, int
                 // other CTAs wrote the operand through the generic proxy; TMA reads through the async proxy
                 fence_proxy_async_all();
             }
-            if (c.p == PH_FC && lane < a.B) {
-                int id;
-                if (c.step == 0) id = __ldcg(a.cur_id + lane);
-                else if (a.forced) id = __ldcg(a.forced + (long long)lane * a.k + (c.step - 1));
-                else id = key_index(__ldcg(a.keys + (long long)lane * a.key_stride + (c.step - 1)));
-                my_id = (id < 0 || id >= a.V) ? 0 : id;
-            }
             map_idx = c.p == PH_QKV ? TCM_X_XQ : c.p == PH_O ? TCM_X_ATTN : c.p == PH_GU ? TCM_X_XM
                     : c.p == PH_DOWN ? TCM_X_ACT : TCM_X_FEAT;
+        }
+        const bool emb = c.p == PH_FC && c.kb >= dkb;
+        if (emb && gathered_step != c.step) {
+            if (!wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(c.step * TC_BARS_PER_STEP + TC_SEQ_GATHER + 1), ctl,
+                           a.error_flag, 11))
+                break;
+            fence_proxy_async_all();
+            gathered_step = c.step;
         }
         if (round > 0 && !wait_mbar(saddr(&ctl->empty[slot]), (round - 1) & 1u, ctl, a.error_flag, 10)) break;
         if (poisoned(ctl)) break;
         const uint32_t bar = saddr(&ctl->full[slot]);
         const uint32_t dst = smemB + slot * TC_B_BYTES;
-        if (c.p == PH_FC && c.kb >= dkb) {
-            // embedding half of the fusion FC: rows gathered by token id; remainder rows are zero
-            const int x = (c.kb - dkb) * TC_BK;
-            if (lane < a.B) tma_load_2d(dst + lane * 128, &P.maps.m[TCM_EMBED], x, my_id, bar, pol_x);
-            else if (lane < erows) tma_load_2d(dst + lane * 128, &P.maps.m[TCM_ZERO], 0, 0, bar, pol_x);
-        } else if (lane == 0) {
-            tma_load_2d(dst, &P.maps.m[map_idx], c.kb * TC_BK, 0, bar, pol_x);
-        }
-        __syncwarp();
+        if (emb) tma_load_2d(dst, &P.maps.m[TCM_X_EMB], (c.kb - dkb) * TC_BK, 0, bar, pol_x);
+        else tma_load_2d(dst, &P.maps.m[map_idx], c.kb * TC_BK, 0, bar, pol_x);
         cursor_next(c, a, cta, G);
         if (++slot == TC_STAGES) { slot = 0; ++round; }
     }
-    __syncwarp();
     if (poisoned(ctl)) drain_after_poison();
+}
+
+// Embedding gather of step s (one warp per CTA): once the previous LM head is complete the chosen tokens are
+// known; their embedding rows are copied into the dense operand buffer that the fusion FC reads.  Step 0's rows
+// were copied by the set-up kernel.  Arrives on the gather barrier of the step.
+__device__ void tc_gather(const TcParams& P, TcCtl* ctl, int s, int cta, int G, int lane) {
+    const TcArgs& a = P.a;
+    if (s > 0) {
+        bool ok = true;
+        if (lane == 0)
+            ok = wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)((s - 1) * TC_BARS_PER_STEP + 8), ctl, a.error_flag, 12);
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (ok) {
+            const int upr = a.d >> 3;                    // 16-byte units per row
+            const int total = a.B * upr;
+            for (int i = cta * 32 + lane; i < total; i += G * 32) {
+                const int b = i / upr, off = i - b * upr;
+                int id = a.forced ? __ldcg(a.forced + (long long)b * a.k + (s - 1))
+                                  : key_index(__ldcg(a.keys + (long long)b * a.key_stride + (s - 1)));
+                if (id < 0 || id >= a.V) id = 0;
+                const uint4 w = ld_stream((const uint4*)(a.embed + (long long)id * a.d) + off);
+                __stcg((uint4*)(a.xe_h + (long long)b * a.d) + off, w);
+            }
+        }
+    }
+    __syncwarp();
+    if (lane == 0) {
+        fence_proxy_async_all();
+        red_release_add_u64(a.bar_counter, 1ull);
+    }
+    __syncwarp();
 }
 
 // ---- MMA issuer ----------------------------------------------------------------------------------
@@ -599,8 +622,9 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
     // the phase that is implied (its operand tiles were loaded after that barrier); without work, wait for it.
     named_sync(TC_BAR_EPI, TC_EPI_THREADS);
     if (etid == 0) {
-        const int need = need_seq(s, p);
-        if (lo == hi && need >= 0)
+        // (the FC phase follows the gather barrier of its step, which its hidden-half operand does not imply)
+        const int need = p == PH_FC ? s * TC_BARS_PER_STEP + TC_SEQ_GATHER : need_seq(s, p);
+        if ((lo == hi || p == PH_FC) && need >= 0)
             wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(need + 1), ctl, a.error_flag, 8);
         fence_proxy_async_all();
         red_release_add_u64(a.bar_counter, 1ull);
@@ -651,10 +675,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
         if (lane == 0) tc_mma_issuer(P, ctl, smemA, smemB, cta, G);
         __syncwarp();
     } else if (warp == 2) {
-        tc_producer_x(P, ctl, smemB, cta, G, lane);
-    } else if (warp >= 4) {
-        // warps 4..7: epilogue of every GEMM phase, and the attention between the QKV and O phases
-        const int etid = tid - 128;
+        if (lane == 0) tc_producer_x(P, ctl, smemB, cta, G);
+        __syncwarp();
+    } else {
+        // warps 4..7: epilogue of every GEMM phase; warp 3: the embedding gather; warps 3..7: the attention
+        // between the QKV and O phases
+        const int atid = tid - 96;
+        const bool is_epi = warp >= 4;
         const int w4 = warp - 4;
         unsigned seg_cnt = 0;
         AttnWArgs aw;
@@ -663,26 +690,31 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
         aw.B = a.B; aw.scale = a.scale; aw.part_acc = a.part_acc; aw.part_ml = a.part_ml; aw.nslot = a.attn_nslot;
         aw.counters = a.counters; aw.attn = a.attn; aw.attn_h = a.attn_h; aw.lo_rows = a.lo ? a.B : 0;
         for (int s = 0; s < a.k; ++s) {
-            tc_epilogue_phase(P, ctl, s, PH_FC, seg_cnt, cta, G, w4, lane);
-            tc_epilogue_phase(P, ctl, s, PH_QKV, seg_cnt, cta, G, w4, lane);
+            if (is_epi) {
+                tc_epilogue_phase(P, ctl, s, PH_FC, seg_cnt, cta, G, w4, lane);
+                tc_epilogue_phase(P, ctl, s, PH_QKV, seg_cnt, cta, G, w4, lane);
+            } else {
+                tc_gather(P, ctl, s, cta, G, lane);
+            }
             // ---- attention: needs every CTA's QKV rows
-            if (etid == 0)
-                wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(s * TC_BARS_PER_STEP + 2), ctl, a.error_flag, 7);
-            named_sync(TC_BAR_EPI, TC_EPI_THREADS);
+            if (atid == 0)
+                wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(s * TC_BARS_PER_STEP + TC_SEQ_ATTN), ctl, a.error_flag, 7);
+            named_sync(TC_BAR_ATT, TC_ATT_WARPS * 32);
             if (!poisoned(ctl)) {
                 aw.step = s;
-                attn_warp_phase<DH, GQ>(aw, cta * TC_ATT_WARPS + w4, G * TC_ATT_WARPS, lane);
+                attn_warp_phase<DH, GQ>(aw, cta * TC_ATT_WARPS + (warp - 3), G * TC_ATT_WARPS, lane);
             }
-            __threadfence();
-            named_sync(TC_BAR_EPI, TC_EPI_THREADS);
-            if (etid == 0) {
+            named_sync(TC_BAR_ATT, TC_ATT_WARPS * 32);
+            if (atid == 0) {
                 fence_proxy_async_all();
                 red_release_add_u64(a.bar_counter, 1ull);
             }
-            tc_epilogue_phase(P, ctl, s, PH_O, seg_cnt, cta, G, w4, lane);
-            tc_epilogue_phase(P, ctl, s, PH_GU, seg_cnt, cta, G, w4, lane);
-            tc_epilogue_phase(P, ctl, s, PH_DOWN, seg_cnt, cta, G, w4, lane);
-            tc_epilogue_phase(P, ctl, s, PH_LM, seg_cnt, cta, G, w4, lane);
+            if (is_epi) {
+                tc_epilogue_phase(P, ctl, s, PH_O, seg_cnt, cta, G, w4, lane);
+                tc_epilogue_phase(P, ctl, s, PH_GU, seg_cnt, cta, G, w4, lane);
+                tc_epilogue_phase(P, ctl, s, PH_DOWN, seg_cnt, cta, G, w4, lane);
+                tc_epilogue_phase(P, ctl, s, PH_LM, seg_cnt, cta, G, w4, lane);
+            }
         }
     }
     tc_fence_before();
@@ -697,7 +729,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
 // ------------------------------------------------------------------------------------------ set-up kernel
 __global__ void tc_setup_kernel(SlotList sl, int k, int d, int lo, int* d_slots, int* d_pos0, int* kv_len,
                                 const float* pend_feat, const int* pend_id, float* feat, bf16* feat_h, int* cur_id,
-                                u64* keys, int key_stride) {
+                                u64* keys, int key_stride, const bf16* embed, int vocab, bf16* xe_h) {
     const int b = blockIdx.x, slot = sl.slot[b];
     if (threadIdx.x == 0) {
         d_slots[b] = slot;
@@ -714,12 +746,17 @@ __global__ void tc_setup_kernel(SlotList sl, int k, int d, int lo, int* d_slots,
         feat_h[(long long)b * d + i] = hi;
         if (lo) feat_h[(long long)(b + sl.n) * d + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
     }
+    // embedding row of the pending token: the fusion FC's embedding operand of step 0
+    int id = pend_id[slot];
+    if (id < 0 || id >= vocab) id = 0;
+    for (int i = threadIdx.x; i < (d >> 3); i += blockDim.x)
+        ((uint4*)(xe_h + (long long)b * d))[i] = ((const uint4*)(embed + (long long)id * d))[i];
 }
 cudaError_t launch_tc_setup(const SlotList& sl, int k, int d, int lo, int* d_slots, int* d_pos0, int* kv_len,
                             const float* pend_feat, const int* pend_id, float* feat, bf16* feat_h, int* cur_id,
-                            u64* keys, int key_stride, cudaStream_t st) {
+                            u64* keys, int key_stride, const bf16* embed, int vocab, bf16* xe_h, cudaStream_t st) {
     tc_setup_kernel<<<sl.n, 256, 0, st>>>(sl, k, d, lo, d_slots, d_pos0, kv_len, pend_feat, pend_id, feat, feat_h,
-                                          cur_id, keys, key_stride);
+                                          cur_id, keys, key_stride, embed, vocab, xe_h);
     return cudaGetLastError();
 }
 
@@ -773,9 +810,9 @@ int tc_max_tiles(const ChainPhase* ph) {
 
 int tc_barriers_per_step() { return TC_BARS_PER_STEP; }
 
-cudaError_t tc_build_maps(TcMaps* maps, const ChainPhase* ph, int d, int qw, int F, int V, const void* embed,
+cudaError_t tc_build_maps(TcMaps* maps, const ChainPhase* ph, int d, int qw, int F,
                           const bf16* feat_h, const bf16* xq_h, const bf16* attn_h, const bf16* xm_h,
-                          const bf16* act_h, const bf16* zero_row) {
+                          const bf16* act_h, const bf16* xe_h) {
     static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
     cudaError_t e;
     for (int p = 0; p < PH_COUNT; ++p) {
@@ -788,9 +825,7 @@ cudaError_t tc_build_maps(TcMaps* maps, const ChainPhase* ph, int d, int qw, int
         e = encode_map(maps->m[ops[i].idx], ops[i].base, TC_OP_ROWS, ops[i].cols, TC_TN, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
         if (e != cudaSuccess) return e;
     }
-    e = encode_map(maps->m[TCM_EMBED], embed, V, d, 1, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
-    if (e != cudaSuccess) return e;
-    return encode_map(maps->m[TCM_ZERO], zero_row, 1, d, 1, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+    return encode_map(maps->m[TCM_X_EMB], xe_h, TC_OP_ROWS, d, TC_TN, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
 }
 
 template <int DH, int GQ>
