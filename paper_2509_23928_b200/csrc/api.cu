@@ -49,6 +49,7 @@ struct hivis_ctx {
     int* tile_ctr;
     int tc_tiles;
     bf16* xe_h;
+    float2* rope_tab;
     int *slot_of, *row_of;
     long long map_cap;
     // host mirrors
@@ -288,7 +289,8 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
          dalloc(c, &c->part_ml, R * cfg->n_q_heads * (long long)c->nsplit_cap * 2) &&
          dalloc(c, &c->counters, R * cfg->n_q_heads) && dalloc(c, &c->bar_counter, 1) &&
          dalloc(c, &c->error_flag, 1) && dalloc(c, &c->slot_of, c->map_cap) &&
-         dalloc(c, &c->row_of, c->map_cap) && dalloc(c, &c->xe_h, R * d);
+         dalloc(c, &c->row_of, c->map_cap) && dalloc(c, &c->xe_h, R * d) &&
+         dalloc(c, &c->rope_tab, 2 * 16 * (cfg->head_dim / 2));
     if (!ok) {
         free_all(c);
         delete c;
@@ -607,7 +609,7 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
         a.keys = c->keys; a.key_stride = c->key_stride;
         a.u = c->u; a.qkv = c->qkv; a.attn = c->attn; a.y = c->y; a.feat = c->feat;
         a.feat_h = c->feat_h; a.xq_h = c->xq; a.attn_h = c->attn_h; a.xm_h = c->xm; a.act_h = c->act_h;
-        a.xe_h = c->xe_h; a.embed = (const bf16*)c->embed;
+        a.xe_h = c->xe_h; a.embed = (const bf16*)c->embed; a.rope_tab = c->rope_tab;
         a.ssq1 = c->ssq1; a.ssq2 = c->ssq2; a.logits_out = out_logits;
         a.partial = c->tc_partial; a.tile_ctr = c->tile_ctr;
         a.Kc = c->Kc; a.Vc = c->Vc; a.inv_freq = c->inv_freq; a.part_acc = c->part_acc; a.part_ml = c->part_ml;

@@ -28,7 +28,7 @@ struct AttnWArgs {
     const int* slots;       // [B]
     const int* pos0;        // [B] cache row of draft step 0
     int step;
-    const double* inv_freq; // [dh/2]
+    const float2* rope_tab; // [B][dh/2] (cos, sin) of every sequence's new position at this step
     int Hq, Hkv, max_len, B;
     float scale;
     float* part_acc;        // [B][Hq][nslot][dh]
@@ -88,7 +88,19 @@ __device__ void attn_warp_phase(const AttnWArgs& a, int gw, int NW, int lane) {
 
     // units of the batch
     unsigned U = 0;
-    for (int b = 0; b < a.B; ++b) U += (unsigned)HG * (unsigned)((__ldg(a.pos0 + b) + a.step + 1 + 31) >> 5);
+    bool uniform = true;
+    const int nb_first = (__ldg(a.pos0) + a.step + 1 + 31) >> 5;
+    for (int b = 0; b < a.B; ++b) {
+        const int nbb = (__ldg(a.pos0 + b) + a.step + 1 + 31) >> 5;
+        U += (unsigned)HG * (unsigned)nbb;
+        uniform = uniform && nbb == nb_first;
+    }
+    // When every key has the same number of blocks and there are at least as many warps as keys, use a whole
+    // number of warps per key: the ranges then start on key boundaries and (with one warp per key) nothing is
+    // published or merged.  Otherwise all warps take equal ranges of the unit list.
+    const int nkeys = a.B * HG;
+    if (uniform && nkeys <= NW) NW = nkeys * (NW / nkeys);
+    if (gw >= NW) return;
     const unsigned u0 = attw_lo(U, gw, NW), u1 = attw_lo(U, gw + 1, NW);
     if (u0 >= u1) return;
 
@@ -119,20 +131,25 @@ __device__ void attn_warp_phase(const AttnWArgs& a, int gw, int NW, int lane) {
         if (fresh) {
             // rotation of this lane's slice [8c, 8c+8) at position p (the same for every head), then the slice
             // of every query head of the group, rotated and scaled
+            {
+                const float4* tab = (const float4*)(a.rope_tab + (long long)b * HALF + ((8 * c) & (HALF - 1)));
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const int d = 8 * c + e;
-                rope_cs(p, a.inv_freq[d < HALF ? d : d - HALF], cs8[e], sn8[e]);
+                for (int e2 = 0; e2 < 4; ++e2) {
+                    const float4 t = __ldcg(tab + e2);
+                    cs8[2 * e2] = t.x; sn8[2 * e2] = t.y; cs8[2 * e2 + 1] = t.z; sn8[2 * e2 + 1] = t.w;
+                }
             }
+            const bool lower = 8 * c < HALF;                  // this slice lies in the first half of the head
 #pragma unroll
             for (int g = 0; g < GQ; ++g) {
                 const float* q = qkv + (h0 + g) * DH;
+                const float4 x0 = __ldcg((const float4*)(q + 8 * c)), x1 = __ldcg((const float4*)(q + 8 * c) + 1);
+                const float4 y0 = __ldcg((const float4*)(q + ((8 * c) ^ HALF))), y1 = __ldcg((const float4*)(q + ((8 * c) ^ HALF)) + 1);
+                const float xs[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+                const float ys[8] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w};
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const int d = 8 * c + e;
-                    const float x = __ldcg(q + d), y = __ldcg(q + (d < HALF ? d + HALF : d - HALF));
-                    qf[g][e] = (d < HALF ? x * cs8[e] - y * sn8[e] : x * cs8[e] + y * sn8[e]) * a.scale;
-                }
+                for (int e = 0; e < 8; ++e)
+                    qf[g][e] = (lower ? xs[e] * cs8[e] - ys[e] * sn8[e] : xs[e] * cs8[e] + ys[e] * sn8[e]) * a.scale;
                 m_run[g] = -INFINITY;
                 l_run[g] = 0.f;
 #pragma unroll
@@ -149,19 +166,32 @@ __device__ void attn_warp_phase(const AttnWArgs& a, int gw, int NW, int lane) {
         float knew[8];
         if (has_new) {
             const bool writer = (h0 % G) == 0 && hrow == 0;      // one key per KV head appends the row
+            const bool lower = 8 * c < HALF;
             const float* kx = qkv + qw + kvh * DH;
+            const float4 x0 = __ldcg((const float4*)(kx + 8 * c)), x1 = __ldcg((const float4*)(kx + 8 * c) + 1);
+            const float4 y0 = __ldcg((const float4*)(kx + ((8 * c) ^ HALF))), y1 = __ldcg((const float4*)(kx + ((8 * c) ^ HALF)) + 1);
+            const float xs[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+            const float ys[8] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w};
+            unsigned pk[4];
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-                const int d = 8 * c + e;
-                const float x = __ldcg(kx + d), y = __ldcg(kx + (d < HALF ? d + HALF : d - HALF));
-                const bf16 kb = __float2bfloat16_rn(d < HALF ? x * cs8[e] - y * sn8[e] : x * cs8[e] + y * sn8[e]);
+                const bf16 kb = __float2bfloat16_rn(lower ? xs[e] * cs8[e] - ys[e] * sn8[e] : xs[e] * cs8[e] + ys[e] * sn8[e]);
                 knew[e] = __bfloat162float(kb);
-                if (writer) Kbase[(long long)p * DH + d] = kb;
+                const unsigned bits = (unsigned)__bfloat16_as_ushort(kb);
+                if (e & 1) pk[e >> 1] |= bits << 16; else pk[e >> 1] = bits;
             }
             if (writer) {
-                const float* vx = qkv + qw + kvw + kvh * DH;
+                *(uint4*)(Kbase + (long long)p * DH + 8 * c) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                const float* vx = qkv + qw + kvw + kvh * DH + 8 * c;
+                const float4 v0 = __ldcg((const float4*)vx), v1 = __ldcg((const float4*)vx + 1);
+                const float vs[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+                unsigned pv[4];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) Vbase[(long long)p * DH + 8 * c + e] = __float2bfloat16_rn(__ldcg(vx + 8 * c + e));
+                for (int e = 0; e < 8; ++e) {
+                    const unsigned bits = (unsigned)__bfloat16_as_ushort(__float2bfloat16_rn(vs[e]));
+                    if (e & 1) pv[e >> 1] |= bits << 16; else pv[e >> 1] = bits;
+                }
+                *(uint4*)(Vbase + (long long)p * DH + 8 * c) = make_uint4(pv[0], pv[1], pv[2], pv[3]);
             }
         }
         // ---- all loads of the unit go out first: the K slices of this lane's rows and (for VPRE rows) this

@@ -171,6 +171,7 @@ struct TcArgs {
     int* tile_ctr;             // arrival counters of split tiles, zero between phases
     void *Kc, *Vc;
     const double* inv_freq;
+    float2* rope_tab;          // [2][16][dh/2] (cos, sin) per sequence at the current step, halves alternate
     float *part_acc, *part_ml;
     int* counters;
     int attn_nslot;            // partial slots per (sequence, head): >= 32-row blocks of the longest sequence

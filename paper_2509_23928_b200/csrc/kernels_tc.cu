@@ -346,6 +346,18 @@ __device__ void tc_producer_x(const TcParams& P, TcCtl* ctl, uint32_t smemB, int
 // were copied by the set-up kernel.  Arrives on the gather barrier of the step.
 __device__ void tc_gather(const TcParams& P, TcCtl* ctl, int s, int cta, int G, int lane) {
     const TcArgs& a = P.a;
+    {
+        // (cos, sin) of every sequence's new position at this step, for the attention of this step; the two
+        // halves of the table alternate between steps, since CTAs still in the previous attention read the other
+        const int half = a.dh >> 1;
+        float2* tab = a.rope_tab + (long long)(s & 1) * 16 * half;
+        for (int i = cta * 32 + lane; i < a.B * half; i += G * 32) {
+            const int b = i / half, f = i - b * half;
+            float cs, sn;
+            rope_cs(__ldg(a.pos0 + b) + s, a.inv_freq[f], cs, sn);
+            __stcg(tab + (long long)b * half + f, make_float2(cs, sn));
+        }
+    }
     if (s > 0) {
         bool ok = true;
         if (lane == 0)
@@ -686,7 +698,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
         unsigned seg_cnt = 0;
         AttnWArgs aw;
         aw.qkv = a.qkv; aw.ld = a.qw + 2 * a.kvw; aw.Kc = (bf16*)a.Kc; aw.Vc = (bf16*)a.Vc; aw.slots = a.slots;
-        aw.pos0 = a.pos0; aw.step = 0; aw.inv_freq = a.inv_freq; aw.Hq = a.Hq; aw.Hkv = a.Hkv; aw.max_len = a.max_len;
+        aw.pos0 = a.pos0; aw.step = 0; aw.rope_tab = a.rope_tab; aw.Hq = a.Hq; aw.Hkv = a.Hkv; aw.max_len = a.max_len;
         aw.B = a.B; aw.scale = a.scale; aw.part_acc = a.part_acc; aw.part_ml = a.part_ml; aw.nslot = a.attn_nslot;
         aw.counters = a.counters; aw.attn = a.attn; aw.attn_h = a.attn_h; aw.lo_rows = a.lo ? a.B : 0;
         for (int s = 0; s < a.k; ++s) {
@@ -702,6 +714,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
             named_sync(TC_BAR_ATT, TC_ATT_WARPS * 32);
             if (!poisoned(ctl)) {
                 aw.step = s;
+                aw.rope_tab = a.rope_tab + (long long)(s & 1) * 16 * (DH / 2);
                 attn_warp_phase<DH, GQ>(aw, cta * TC_ATT_WARPS + (warp - 3), G * TC_ATT_WARPS, lane);
             }
             named_sync(TC_BAR_ATT, TC_ATT_WARPS * 32);
