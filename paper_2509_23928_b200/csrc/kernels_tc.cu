@@ -466,12 +466,16 @@ __device__ void epi_output(const TcArgs& a, TcCtl* ctl, int p, int s, int tile, 
         float* ssq = p == PH_FC ? a.ssq1 : a.ssq2;
         const float g = rok ? __bfloat162float(gamma[row]) : 0.f;
         const float add0 = (rok && rho) ? rho[row] : 0.f;
+        // the addends of all sequences are requested before any store (stores would order the loads behind them)
+        float add[16];
+#pragma unroll
+        for (int b = 0; b < 16; ++b) add[b] = (p == PH_O && rok && b < B) ? __ldcg(a.u + (long long)b * N + row) : add0;
 #pragma unroll
         for (int b = 0; b < 16; ++b) {
             if (b >= B) break;
             float r = 0.f;
             if (rok) {
-                r = val[b] + (p == PH_FC ? add0 : __ldcg(a.u + (long long)b * N + row));
+                r = val[b] + add[b];
                 outf[(long long)b * N + row] = r;
                 store_operand(outh, N, b, row, g * r, lo_rows);
             }
@@ -505,10 +509,13 @@ __device__ void epi_output(const TcArgs& a, TcCtl* ctl, int p, int s, int tile, 
         }
     } else if (p == PH_DOWN) {
         if (rok) {
+            float add[16];
+#pragma unroll
+            for (int b = 0; b < 16; ++b) add[b] = b < B ? __ldcg(a.y + (long long)b * N + row) : 0.f;
 #pragma unroll
             for (int b = 0; b < 16; ++b) {
                 if (b >= B) break;
-                const float r = __ldcg(a.y + (long long)b * N + row) + val[b];
+                const float r = add[b] + val[b];
                 a.feat[(long long)b * N + row] = r;
                 store_operand(a.feat_h, N, b, row, r, lo_rows);
             }
