@@ -422,6 +422,29 @@ __device__ void tc_mma_issuer(const TcParams& P, TcCtl* ctl, uint32_t smemA, uin
 }
 
 // ---- output stages ---------------------------------------------------------------------------------
+// Transposing butterfly: every lane holds 16 values (one per batch column); afterwards lane L holds the
+// reduction over all 32 lanes of column warp_col16(L) (lanes L and L^1 hold the same column).  16 shuffles
+// instead of 16 x 5, and they are independent of each other.
+__device__ __forceinline__ int warp_col16(int lane) {
+    return 8 * ((lane >> 4) & 1) + 4 * ((lane >> 3) & 1) + 2 * ((lane >> 2) & 1) + ((lane >> 1) & 1);
+}
+template <typename T, typename Op>
+__device__ __forceinline__ T warp_reduce16(T (&v)[16], int lane, Op op) {
+#pragma unroll
+    for (int off = 16, n = 8; off >= 2; off >>= 1, n >>= 1) {
+        const bool up = (lane & off) != 0;
+#pragma unroll
+        for (int t = 0; t < n; ++t) {
+            const T send = up ? v[t] : v[t + n];
+            const T keep = up ? v[t + n] : v[t];
+            v[t] = op(keep, __shfl_xor_sync(0xffffffffu, send, off));
+        }
+    }
+    return op(v[0], __shfl_xor_sync(0xffffffffu, v[0], 1));
+}
+struct OpAdd { __device__ __forceinline__ float operator()(float x, float y) const { return x + y; } };
+struct OpMaxU64 { __device__ __forceinline__ u64 operator()(u64 x, u64 y) const { return x > y ? x : y; } };
+
 __device__ __forceinline__ void store_operand(bf16* buf, int width, int b, int col, float x, int lo_rows) {
     const bf16 hi = __float2bfloat16_rn(x);
     buf[(long long)b * width + col] = hi;
@@ -470,20 +493,20 @@ __device__ void epi_output(const TcArgs& a, TcCtl* ctl, int p, int s, int tile, 
         float add[16];
 #pragma unroll
         for (int b = 0; b < 16; ++b) add[b] = (p == PH_O && rok && b < B) ? __ldcg(a.u + (long long)b * N + row) : add0;
+        float sq[16];
 #pragma unroll
         for (int b = 0; b < 16; ++b) {
-            if (b >= B) break;
             float r = 0.f;
-            if (rok) {
+            if (rok && b < B) {
                 r = val[b] + add[b];
                 outf[(long long)b * N + row] = r;
                 store_operand(outh, N, b, row, g * r, lo_rows);
             }
-            float sq = r * r;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-            if (lane == 0) ssq[(long long)(tile * 4 + w4) * 16 + b] = sq;
+            sq[b] = r * r;
         }
+        const float tot = warp_reduce16(sq, lane, OpAdd());
+        const int col = warp_col16(lane);
+        if ((lane & 1) == 0 && col < B) ssq[(long long)(tile * 4 + w4) * 16 + col] = tot;
     } else if (p == PH_QKV) {
         const float bias = (rok && a.bqkv) ? __bfloat162float(a.bqkv[row]) : 0.f;
         if (rok) {
@@ -521,18 +544,18 @@ __device__ void epi_output(const TcArgs& a, TcCtl* ctl, int p, int s, int tile, 
             }
         }
     } else {   // PH_LM
+        u64 keys[16];
 #pragma unroll
         for (int b = 0; b < 16; ++b) {
-            if (b >= B) break;
-            if (rok && a.logits_out) a.logits_out[((long long)b * a.k + s) * a.V + row] = val[b];
-            u64 key = rok ? pack_key(val[b], row) : 0ull;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                const u64 other = __shfl_xor_sync(0xffffffffu, key, o);
-                key = other > key ? other : key;
+            keys[b] = 0ull;
+            if (rok && b < B) {
+                if (a.logits_out) a.logits_out[((long long)b * a.k + s) * a.V + row] = val[b];
+                keys[b] = pack_key(val[b], row);
             }
-            if (lane == 0 && key) atomicMax(a.keys + (long long)b * a.key_stride + s, key);
         }
+        const u64 best = warp_reduce16(keys, lane, OpMaxU64());
+        const int col = warp_col16(lane);
+        if ((lane & 1) == 0 && col < B && best) atomicMax(a.keys + (long long)col * a.key_stride + s, best);
     }
 }
 
@@ -546,6 +569,21 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
     const long long lo = range_lo(sh.W, cta, G), hi = range_lo(sh.W, cta + 1, G);
     long long idx = lo;
     bool need_scale = (p == PH_QKV || p == PH_GU);
+    // Contributors of the (at most two) tiles this CTA shares with others, worked out while the first
+    // accumulator is still being computed: first contributor, its slot bit, number of contributors.
+    int cinfo[2][3] = {{0, 0, 0}, {0, 0, 0}};
+    if (etid == 0 && lo < hi && sh.W >= G) {
+        const long long tl[2] = {lo / sh.nkb, (hi - 1) / sh.nkb};
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const long long t0 = tl[q] * sh.nkb;
+            const int cf = owner_of(sh.W, G, t0);
+            cinfo[q][0] = cf;
+            cinfo[q][1] = t0 == range_lo(sh.W, cf, G) ? 0 : 1;
+            cinfo[q][2] = owner_of(sh.W, G, t0 + sh.nkb - 1) - cf + 1;
+        }
+    }
+    const int tile_first = (int)(lo / sh.nkb);
     while (idx < hi) {
         const int tile = (int)(idx / sh.nkb), kb0 = (int)(idx % sh.nkb);
         const int n = (int)((hi - idx) < (long long)(sh.nkb - kb0) ? (hi - idx) : (long long)(sh.nkb - kb0));
@@ -572,17 +610,19 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
             if (etid == 0) {
                 // contributors = the CTAs whose (non-empty) ranges meet this tile, in range order; when every
                 // CTA has work in the phase they are consecutive CTAs
-                const long long t0 = (long long)tile * sh.nkb;
-                const int cf = owner_of(sh.W, G, t0);
-                int nc;
+                int cf, fs, nc;
                 if (sh.W >= G) {
-                    nc = owner_of(sh.W, G, t0 + sh.nkb - 1) - cf + 1;
+                    const int q = tile == tile_first ? 0 : 1;
+                    cf = cinfo[q][0]; fs = cinfo[q][1]; nc = cinfo[q][2];
                 } else {
+                    const long long t0 = (long long)tile * sh.nkb;
+                    cf = owner_of(sh.W, G, t0);
+                    fs = t0 == range_lo(sh.W, cf, G) ? 0 : 1;
                     nc = 0;
                     for (long long i = t0; i < t0 + sh.nkb; ++nc) i = range_lo(sh.W, owner_of(sh.W, G, i) + 1, G);
                 }
                 ctl->c_first = cf;
-                ctl->c_first_slot = t0 == range_lo(sh.W, cf, G) ? 0 : 1;
+                ctl->c_first_slot = fs;
                 ctl->n_contrib = nc;
                 __threadfence();                       // the CTA's partial (ordered before by the barrier) is visible first
                 const int old = atomicAdd(a.tile_ctr + tile, 1);
