@@ -27,6 +27,12 @@ if ROOT not in sys.path:
 
 import hivis_inputs as hi  # noqa: E402
 
+# DRAM bytes (read + written) of ONE launch of the chain kernel, from the ncu captures summarised under
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum).  Keyed by workload; a workload without a capture,
+# or a kernel that changed since, reports null.
+NCU_TRAFFIC = {"c2_llava_b1": 3672459000 + 4513280, "c5a_llava_b16_text_only": 3732648000 + 7567104,
+               "c4_qwen_b8": 11267649280 + 29625856}
+
 METRIC = "draft_steps_per_s"
 UNIT = "draft steps/s"
 
@@ -272,7 +278,8 @@ def main():
         dom = max((n for n in kern), key=lambda n: prof[n][0])
         dom_bytes = class_bytes[dom]
     roofline = {"bound": "hbm", "kernel": dom, "achieved": kern[dom]["GBps"], "peak": peak, "unit": "GB/s",
-                "frac": round(kern[dom]["GBps"] / peak, 4), "peak_kind": peak_kind, "traffic": None,
+                "frac": round(kern[dom]["GBps"] / peak, 4), "peak_kind": peak_kind,
+                "traffic": NCU_TRAFFIC.get(wl.name) if (dom == "draft_chain" and world == 1) else None,
                 "algorithmic_bytes_per_launch": dom_bytes, "per_kernel": kern}
 
     draft_us_per_step = float(np.median(draft_ms)) / k * 1e3
