@@ -180,8 +180,14 @@ int hivis_debug_tap(hivis_ctx* ctx, int which, float* out, void* stream);
  * runs all k steps in one persistent cooperative kernel that streams the weights with TMA and multiplies
  * on the tcgen05 tensor cores (weights as the M operand, batch as N); 2 = use it for one sequence as well;
  * 0 = never.  What neither kernel takes runs as separate kernel launches per step.  All paths give the
- * same results up to fp32 summation order and the bf16 rounding of the tensor-core operand.            */
-enum { HIVIS_OPT_CHAIN_KERNEL = 0, HIVIS_OPT_TC_KERNEL = 1 };
+ * same results up to fp32 summation order and the bf16 rounding of the tensor-core operand.
+ * HIVIS_OPT_WAIT_LIMIT_US (default 1 000 000): how long a device-side wait of the chain kernels (grid
+ * barrier, copy completion) may last before the kernel gives up, raises the error word that hivis_status
+ * reports and returns in an orderly way.
+ * HIVIS_OPT_DEBUG_MISS_BARRIER (test aid): 1 makes the grid barriers of the NEXT hivis_draft call
+ * impossible to complete, so that every wait runs into its limit: hivis_status then returns
+ * HIVIS_ERR_TIMEOUT and the context is usable again.  Nothing faults or hangs.                          */
+enum { HIVIS_OPT_CHAIN_KERNEL = 0, HIVIS_OPT_TC_KERNEL = 1, HIVIS_OPT_WAIT_LIMIT_US = 2, HIVIS_OPT_DEBUG_MISS_BARRIER = 3 };
 int hivis_set_option(hivis_ctx* ctx, int option, int value);
 
 /* Synchronises `stream` and reports whether any kernel since the last call gave up on a bounded

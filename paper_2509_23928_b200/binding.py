@@ -20,6 +20,8 @@ EXPORTS = ("hivis_init", "hivis_destroy", "hivis_prefill", "hivis_draft", "hivis
            "hivis_status", "hivis_verify_noalloc")
 HIVIS_OPT_CHAIN_KERNEL = 0
 HIVIS_OPT_TC_KERNEL = 1
+HIVIS_OPT_WAIT_LIMIT_US = 2
+HIVIS_OPT_DEBUG_MISS_BARRIER = 3
 PROFILE_CLASSES = ("fuse_fc", "qkv", "attention", "o_proj", "gate_up", "down", "lm_head_argmax", "setup_finish",
                    "draft_chain")
 
@@ -289,6 +291,13 @@ class Drafter:
         """False/0: never; True: for every batch size it supports (2 in the C API); "auto"/1: the default."""
         v = 1 if on == "auto" else (2 if on is True else int(on))
         hivis_set_option(self.ctx, HIVIS_OPT_TC_KERNEL, v)
+
+    def set_wait_limit_us(self, us: int):
+        hivis_set_option(self.ctx, HIVIS_OPT_WAIT_LIMIT_US, int(us))
+
+    def miss_next_barrier(self):
+        """Test aid: the grid barriers of the next draft cannot complete, so its waits run out."""
+        hivis_set_option(self.ctx, HIVIS_OPT_DEBUG_MISS_BARRIER, 1)
 
     def status(self):
         hivis_status(self.ctx)

@@ -43,6 +43,8 @@ struct hivis_ctx {
     int* error_flag;
     // tensor-core chain kernel (bf16, up to 16 sequences)
     bool tc_ok;                   // cooperative launch available, shapes supported, tensor maps built
+    long long wait_cycles;        // option HIVIS_OPT_WAIT_LIMIT_US, in cycles
+    bool debug_skew;              // option HIVIS_OPT_DEBUG_MISS_BARRIER: the next draft's grid barriers cannot complete
     int opt_tc;                   // option HIVIS_OPT_TC_KERNEL: 0 off, 1 for two or more sequences, 2 always
     TcMaps tc_maps;
     float* tc_partial;
@@ -247,6 +249,8 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
     c->opt_chain = true;
     c->chain_ok = false;
     c->opt_tc = 1;
+    c->wait_cycles = 2000000000ll;
+    c->debug_skew = false;
     c->tc_ok = false;
     c->tc_partial = nullptr;
     c->tile_ctr = nullptr;
@@ -578,7 +582,9 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
         a.logits_out = out_logits;
         a.out_ids = out_ids;
         plan_attention(c, max_rows, c->num_sms / g.n_q_heads, &a.attn_chunk, &a.attn_nsplit);
-        a.bar_base = c->bar_count_host;
+        a.bar_base = c->bar_count_host + (c->debug_skew ? (1ull << 40) : 0ull);
+        a.wait_cycles = c->wait_cycles;
+        c->debug_skew = false;
         CKP(c, CLS_CHAIN, st, launch_draft_chain(a, c->dtype, c->num_sms, st));
         c->bar_count_host += (u64)c->num_sms * (u64)(chain_barriers_per_step() * k);
         const int s0 = sl.slot[0];
@@ -615,7 +621,9 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
         a.Kc = c->Kc; a.Vc = c->Vc; a.inv_freq = c->inv_freq; a.part_acc = c->part_acc; a.part_ml = c->part_ml;
         a.counters = c->counters;
         a.attn_nslot = c->nsplit_cap;
-        a.bar_counter = c->bar_counter; a.bar_base = c->bar_count_host; a.error_flag = c->error_flag;
+        a.bar_counter = c->bar_counter; a.bar_base = c->bar_count_host + (c->debug_skew ? (1ull << 40) : 0ull);
+        a.wait_cycles = c->wait_cycles; a.error_flag = c->error_flag;
+        c->debug_skew = false;
         CKP(c, CLS_CHAIN, st, launch_tc_chain(c->tc_maps, a, c->num_sms, st));
         c->bar_count_host += (u64)c->num_sms * (u64)(tc_barriers_per_step() * k);
         CKP(c, CLS_OTHER, st, launch_draft_finish(B, k, c->keys, c->key_stride, out_ids, st));
@@ -818,6 +826,15 @@ int hivis_set_option(hivis_ctx* c, int option, int value) {
     if (option == HIVIS_OPT_TC_KERNEL) {
         if (value < 0 || value > 2) return fail(c, HIVIS_ERR_ARG, "HIVIS_OPT_TC_KERNEL takes 0, 1 or 2");
         c->opt_tc = value;
+        return HIVIS_OK;
+    }
+    if (option == HIVIS_OPT_WAIT_LIMIT_US) {
+        if (value < 100 || value > 10000000) return fail(c, HIVIS_ERR_ARG, "wait limit %d us outside [100, 10000000]", value);
+        c->wait_cycles = (long long)value * 2000ll;          // at most ~2 GHz
+        return HIVIS_OK;
+    }
+    if (option == HIVIS_OPT_DEBUG_MISS_BARRIER) {
+        c->debug_skew = value != 0;
         return HIVIS_OK;
     }
     return fail(c, HIVIS_ERR_ARG, "unknown option %d", option);

@@ -119,6 +119,7 @@ struct ChainArgs {
     int attn_chunk, attn_nsplit;
     u64* bar_counter;          // arrival counter of the grid barrier, only ever incremented
     u64 bar_base;              // its value when this launch starts
+    long long wait_cycles;     // limit of every device-side wait, in SM clock cycles
     int* error_flag;           // set non-zero by a kernel that gave up on a wait
     int off_x, off_part, off_bar, off_misc;   // shared-memory layout, filled by the launcher
 };
@@ -177,6 +178,7 @@ struct TcArgs {
     int attn_nslot;            // partial slots per (sequence, head): >= 32-row blocks of the longest sequence
     u64* bar_counter;
     u64 bar_base;
+    long long wait_cycles;     // limit of every device-side wait, in SM clock cycles
     int* error_flag;
 };
 // fills `maps` for the given buffers; returns cudaSuccess or an error (driver entry point missing, bad shape)

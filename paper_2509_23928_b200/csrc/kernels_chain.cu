@@ -30,7 +30,6 @@
 #ifndef CHAIN_CHUNK_BYTES
 #define CHAIN_CHUNK_BYTES 4096
 #endif
-#define CHAIN_WAIT_CYCLES 2000000000ll      // ~1 s: far beyond any legitimate wait
 
 // ------------------------------------------------------------------------------------------ PTX helpers
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -96,7 +95,7 @@ __device__ __forceinline__ bool grid_barrier(const ChainArgs& a, ChainMisc* misc
         unsigned it = 0;
         bool ok = true;
         while (ld_acquire_u64(a.bar_counter) < target) {
-            if ((++it & 255u) == 0u && (ld_relaxed_int(a.error_flag) != 0 || clock64() - t0 > CHAIN_WAIT_CYCLES)) {
+            if ((++it & 255u) == 0u && (ld_relaxed_int(a.error_flag) != 0 || clock64() - t0 > a.wait_cycles)) {
                 ok = false;
                 break;
             }
@@ -250,7 +249,7 @@ __global__ void __launch_bounds__(CHAIN_THREADS, 1) draft_chain_kernel(const Cha
             if (!mbar_try_wait(bar, parity)) {
                 const long long t0 = clock64();
                 while (!mbar_try_wait(bar, parity)) {
-                    if (clock64() - t0 > CHAIN_WAIT_CYCLES) {
+                    if (clock64() - t0 > a.wait_cycles) {
                         atomicExch(a.error_flag, 2);
                         misc->abort_flag = 1;
                         return false;
@@ -439,7 +438,7 @@ __global__ void __launch_bounds__(CHAIN_THREADS, 1) draft_chain_kernel(const Cha
         const uint32_t parity = (ci / CHAIN_STAGES) & 1u;
         const long long t0 = clock64();
         while (!mbar_try_wait(bar, parity))
-            if (clock64() - t0 > CHAIN_WAIT_CYCLES) break;
+            if (clock64() - t0 > a.wait_cycles) break;
     }
 }
 

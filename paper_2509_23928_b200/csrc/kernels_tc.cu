@@ -47,7 +47,6 @@
 #define TC_BAR_ATT 2
 #define TC_EPI_THREADS 128
 #define TC_BAR_EPI 3
-#define TC_WAIT_CYCLES 2000000000ll      // ~1 s: far beyond any legitimate wait
 #define TC_TMEM_COLS 32
 
 // instruction descriptor of tcgen05.mma kind::f16: fp32 accumulate, bf16 x bf16, both K-major, N=16, M=128
@@ -64,6 +63,7 @@ struct TcCtl {
     u64 full[TC_STAGES], empty[TC_STAGES], tfull[2], tempty[2];
     uint32_t tmem_base;
     int abort_flag;
+    long long wait_cycles;      // limit of every wait
     int last_flag, c_first, c_first_slot, n_contrib;
     float scale[16];
     float red[8][16];
@@ -178,7 +178,7 @@ __device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, TcCtl* 
         if ((++it & 63u) == 0u) {
             if (poisoned(ctl)) return false;
             if (ld_relaxed_int(error_flag) != 0) { *(volatile int*)&ctl->abort_flag = 1; return false; }
-            if (clock64() - t0 > TC_WAIT_CYCLES) { poison(ctl, error_flag, code); return false; }
+            if (clock64() - t0 > ctl->wait_cycles) { poison(ctl, error_flag, code); return false; }
         }
     }
     return true;
@@ -192,7 +192,7 @@ __device__ __forceinline__ bool wait_grid(const u64* counter, u64 target, TcCtl*
         if ((++it & 63u) == 0u) {
             if (poisoned(ctl)) return false;
             if (ld_relaxed_int(error_flag) != 0) { *(volatile int*)&ctl->abort_flag = 1; return false; }
-            if (clock64() - t0 > TC_WAIT_CYCLES) { poison(ctl, error_flag, code); return false; }
+            if (clock64() - t0 > ctl->wait_cycles) { poison(ctl, error_flag, code); return false; }
         }
     }
     return true;
@@ -713,6 +713,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
             mbar_init(saddr(&ctl->tempty[i]), TC_EPI_THREADS);
         }
         ctl->abort_flag = 0;
+        ctl->wait_cycles = a.wait_cycles;
         ctl->last_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async_all();

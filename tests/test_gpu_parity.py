@@ -411,3 +411,39 @@ def test_full_size_c3_llava_b16_ragged_sampled():
 
 def test_full_size_c4_qwen_b8_sampled():
     _sampled_full_size("c4_qwen_b8", 2)
+
+
+@pytest.mark.parametrize("name,tc", [("mini_mha_b1", False), ("mini_mha_b1", True), ("mini_gqa_b16_ragged", True)])
+def test_device_waits_run_out_cleanly_and_context_recovers(name, tc):
+    """Failure detection without a fault: the grid barriers of one draft are made impossible to complete,
+    every device-side wait runs into its (shortened) limit, the kernel returns by itself, hivis_status
+    reports HIVIS_ERR_TIMEOUT, and the same context then drafts correctly again."""
+    import time
+    import torch
+    from paper_2509_23928_b200 import HivisError
+    wl = hi.workload(name)
+    case = Case(wl)
+    try:
+        dr = case.drafter
+        dr.set_tc_kernel(tc)
+        case.gpu_prefill()
+        dr.set_wait_limit_us(2000)
+        dr.miss_next_barrier()
+        t0 = time.perf_counter()
+        dr.draft(wl.batch, wl.k, case.d_resid)
+        torch.cuda.synchronize()
+        assert time.perf_counter() - t0 < 10.0
+        with pytest.raises(HivisError) as e:
+            dr.status()
+        assert e.value.code == -7
+        dr.status()                                       # the error word was cleared
+        dr.set_wait_limit_us(1000000)
+        ref = case.oracle_run()
+        ids_o = np.stack([r["ids"] for r in ref])
+        case.gpu_restore()
+        ids_f, logits_f = case.gpu_draft(forced=ids_o)
+        dr.status()
+        err = row_rel_err(logits_f, np.stack([r["logits"] for r in ref]))
+        assert err.max() <= 2e-2
+    finally:
+        case.close()
