@@ -47,6 +47,27 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def max_over_ranks(value: float, dist, device: str) -> float:
+    """Largest `value` over all ranks (the job's time is the slowest replica's); identity without a group."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(world: int, steps: int, k: int, slowest_ms: float) -> float:
+    """Whole-job draft steps/s of `world` independent replicas that each ran `steps` benchmark steps of k
+    draft steps, timed by the slowest replica."""
+    return world * steps * k / (slowest_ms * 1e-3)
+
+
+def replica_workload(wl, rank: int, world: int):
+    """Replica `rank` of `world`: same shapes, its own seed (no data is shared, no collective on the path)."""
+    return wl if world == 1 else hi.scaled(wl, seed=wl.seed + 100 * rank)
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -170,8 +191,7 @@ def main():
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    if world > 1:
-        wl = hi.scaled(wl, seed=wl.seed + 100 * rank)      # independent replicas, same shapes
+    wl = replica_workload(wl, rank, world)                 # independent replicas, same shapes
 
     # ---------------- set-up (untimed): weights, prompt, prefill
     W = hi.make_weights(wl.dims, wl.seed)
@@ -237,10 +257,7 @@ def main():
     draft_ms = np.array([ev[i][0].elapsed_time(draft_ev[i]) for i in range(args.steps)])
     total_ms = float(step_ms.sum())
     clocks = sampler.stop() if rank == 0 else None
-    if dist is not None:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dist, "cuda")
     ok_planted = bool((acc.cpu().numpy() == planted).all())
 
     # ---------------- per-kernel device time (separate pass: events around every launch)
@@ -316,11 +333,8 @@ def main():
             h_res.copy_(d_res, non_blocking=True)
             torch.cuda.synchronize()
         t_e2e = time.perf_counter() - t0
-        if dist is not None:
-            t = torch.tensor([t_e2e], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            t_e2e = float(t.item())
-        e2e = {"value": world * n_e2e * k / t_e2e, "unit": UNIT,
+        t_e2e = max_over_ranks(t_e2e, dist, "cuda")
+        e2e = {"value": job_throughput(world, n_e2e, k, t_e2e * 1e3), "unit": UNIT,
                "h2d_bytes_per_step": int(h_resid.numel() * h_resid.element_size() + h_logits.numel() * h_logits.element_size()),
                "d2h_bytes_per_step": int(h_ids.numel() * 4 + 3 * B * 4), "steps": n_e2e,
                "ms_per_step": t_e2e / n_e2e * 1e3}
@@ -333,7 +347,7 @@ def main():
         cpu_baseline["us_per_step"] = round(cb["us_per_step"], 1)
 
     if rank == 0:
-        line = {"metric": METRIC, "value": world * args.steps * k / (total_ms * 1e-3), "unit": UNIT,
+        line = {"metric": METRIC, "value": job_throughput(world, args.steps, k, total_ms), "unit": UNIT,
                 "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
                 "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16 storage, f32 accumulate" if D.dtype == "bf16" else "f32",
