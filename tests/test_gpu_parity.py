@@ -27,6 +27,19 @@ def test_draft_kv_verify_parity_small(name, tc):
         case.close()
 
 
+def test_more_sequences_than_the_chain_kernels_take():
+    """20 sequences: beyond the 16 of the tensor-core chain kernel, so the per-phase kernels run in two passes."""
+    wl = hi.scaled(hi.workload("mini_gqa_b16_ragged"), batch=20, k=3, seed=2103)
+    case = Case(wl)
+    try:
+        res = check_draft_parity(case)
+        case.drafter.status()
+        check_kv_parity(case, res["ref"])
+        check_verify_parity(case, res["ids_o"])
+    finally:
+        case.close()
+
+
 def test_c1_ids_exact_and_tight_logits():
     case = Case(hi.workload("c1_tiny_f32_b1"))
     try:
