@@ -37,7 +37,7 @@
 #include "attn_warp.cuh"
 
 #define TC_THREADS 256
-#define TC_STAGES 11
+#define TC_STAGES 12
 #define TC_BK 64
 #define TC_TM 128
 #define TC_TN 16
