@@ -244,8 +244,8 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
     const size_t es = c->esize;
     const long long d = cfg->d, F = cfg->ffn, V = cfg->vocab, R = c->rows_cap, MB = cfg->max_batch;
     c->chunk = 128;
-    c->nsplit_cap = (cfg->max_len + 31) / 32;
-    if (c->nsplit_cap > 512) c->nsplit_cap = 512;
+    c->nsplit_cap = (cfg->max_len + 31) / 32 + 1;       // blocks of 32 rows, and the rows of the running call
+    if (c->nsplit_cap > 513) c->nsplit_cap = 513;
     c->opt_chain = true;
     c->chain_ok = false;
     c->opt_tc = 1;
@@ -357,7 +357,7 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
         fill_chain_args(c, &ca);
         c->chain_ok = chain_smem_bytes(ca, c->dtype, c->num_sms) != 0;
     }
-    if (c->dtype == HIVIS_BF16 && c->num_sms > 0 && c->chain_ok_coop && (cfg->max_len + 31) / 32 <= c->nsplit_cap &&
+    if (c->dtype == HIVIS_BF16 && c->num_sms > 0 && c->chain_ok_coop && (cfg->max_len + 31) / 32 + 1 <= c->nsplit_cap &&
         tc_supported(cfg->d, cfg->head_dim, cfg->n_q_heads, cfg->n_kv_heads, cfg->ffn)) {
         ChainArgs ca;
         fill_chain_args(c, &ca);

@@ -62,6 +62,7 @@ struct TcParams {
 struct TcCtl {
     u64 full[TC_STAGES], empty[TC_STAGES], tfull[2], tempty[2];
     uint32_t tmem_base;
+    unsigned issued;            // ring items the weight producer has armed so far
     int abort_flag;
     long long wait_cycles;      // limit of every wait
     int last_flag, c_first, c_first_slot, n_contrib;
@@ -115,6 +116,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* map, int x
         "[%0], [%1, {%2, %3}], [%4], %5;" ::"r"(dst),
         "l"(map), "r"(x), "r"(y), "r"(bar), "l"(pol)
         : "memory");
+}
+// untiled bulk copy global -> shared (16-byte aligned addresses, size a multiple of 16 bytes)
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
 }
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -175,6 +182,32 @@ __device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, TcCtl* 
     const long long t0 = clock64();
     unsigned it = 0;
     while (!mbar_try(bar, parity)) {
+        if ((++it & 63u) == 0u) {
+            if (poisoned(ctl)) return false;
+            if (ld_relaxed_int(error_flag) != 0) { *(volatile int*)&ctl->abort_flag = 1; return false; }
+            if (clock64() - t0 > ctl->wait_cycles) { poison(ctl, error_flag, code); return false; }
+        }
+    }
+    return true;
+}
+// Wait until the weight producer has armed ring item `idx` (absolute position).  A stage's barrier tells only
+// the parity of its phase, so whoever does not consume the ring strictly in order (the attention warps; the
+// MMA issuer after it stepped over attention items) first makes sure the stage is in the phase it means to
+// wait for: the producer arms item idx only after item idx - TC_STAGES has been handed back.
+__device__ __forceinline__ unsigned ld_acquire_cta_u32(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(saddr(p)) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_cta_u32(unsigned* p, unsigned v) {
+    asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(saddr(p)), "r"(v) : "memory");
+}
+__device__ __forceinline__ bool wait_issued(TcCtl* ctl, unsigned idx, int* error_flag, int code) {
+    if (poisoned(ctl)) return false;
+    if ((int)(ld_acquire_cta_u32(&ctl->issued) - idx) > 0) return true;
+    const long long t0 = clock64();
+    unsigned it = 0;
+    while ((int)(ld_acquire_cta_u32(&ctl->issued) - idx) <= 0) {
         if ((++it & 63u) == 0u) {
             if (poisoned(ctl)) return false;
             if (ld_relaxed_int(error_flag) != 0) { *(volatile int*)&ctl->abort_flag = 1; return false; }
@@ -277,16 +310,127 @@ __device__ __forceinline__ void drain_after_poison() {
     while (clock64() - t1 < 4000000ll) {}
 }
 
+// ---- attention items of the ring -------------------------------------------------------------------
+// The attention of a step takes its prefix blocks through the same ring as the weight tiles: between the
+// QKV tiles and the O tiles of the step the weight producer issues one item per attention unit of this CTA's
+// attention warps, round-robin over the warps (round r: the r-th unit of every warp that has one).  The
+// attention warps consume these items; the MMA issuer and the operand producer step over them.
+struct TcAttInfo {
+    AttwPlan pl;
+    unsigned n[TC_ATT_WARPS];       // units of attention warp w of this CTA (global warp number w * G + cta)
+    unsigned total;
+};
+__device__ __forceinline__ TcAttInfo tc_att_info(const TcArgs& a, int HG, int cta, int G) {
+    TcAttInfo t;
+    t.pl = attw_plan(a.pos0, a.B, HG, G * TC_ATT_WARPS);
+    t.total = 0;
+#pragma unroll
+    for (int w = 0; w < TC_ATT_WARPS; ++w) {
+        unsigned u0, u1;
+        attw_range(t.pl, w * G + cta, u0, u1);
+        t.n[w] = u1 - u0;
+        t.total += t.n[w];
+    }
+    return t;
+}
+__device__ __forceinline__ void ring_skip(unsigned& slot, unsigned& round, unsigned n) {
+    const unsigned t = slot + n;
+    round += t / TC_STAGES;
+    slot = t % TC_STAGES;
+}
+
+// What an attention warp sees of the ring.
+struct TcAttRing {
+    TcCtl* ctl;
+    int* error_flag;
+    uint32_t smemA;
+    unsigned base;                  // ring position of the CTA's first attention item of this step
+    unsigned n[TC_ATT_WARPS];
+    int w;
+    __device__ __forceinline__ unsigned position(unsigned r) const {
+        unsigned idx = base;
+#pragma unroll
+        for (int w2 = 0; w2 < TC_ATT_WARPS; ++w2) idx += (n[w2] < r ? n[w2] : r) + ((w2 < w && n[w2] > r) ? 1u : 0u);
+        return idx;
+    }
+    __device__ __forceinline__ bool acquire(unsigned r, uint32_t& addr) {
+        const unsigned idx = position(r), slot = idx % TC_STAGES, round = idx / TC_STAGES;
+        addr = smemA + slot * TC_A_BYTES;
+        if (!wait_issued(ctl, idx, error_flag, 15)) return false;
+        return wait_mbar(saddr(&ctl->full[slot]), round & 1u, ctl, error_flag, 13);
+    }
+    __device__ __forceinline__ void release(unsigned r) { mbar_arrive(saddr(&ctl->empty[position(r) % TC_STAGES])); }
+};
+
+// One step's attention items (producer thread).  A prefix block is two bulk copies: its K rows to the start
+// of the stage, its V rows behind the room of 32 K rows.  The prefix is not written during the launch, so
+// these copies need no grid barrier.  A tail unit is an item without data.
+template <int DH, int GQ>
+__device__ bool tc_issue_attention(const TcArgs& a, TcCtl* ctl, uint32_t smemA, const AttwCursor (&first)[TC_ATT_WARPS],
+                                   unsigned& slot, unsigned& round) {
+    AttwCursor cur[TC_ATT_WARPS];
+#pragma unroll
+    for (int w = 0; w < TC_ATT_WARPS; ++w) cur[w] = first[w];
+    const int HG = a.Hq / GQ, Gh = a.Hq / a.Hkv;
+    bool any = true;
+    while (any) {
+        any = false;
+#pragma unroll
+        for (int w = 0; w < TC_ATT_WARPS; ++w) {
+            if (cur[w].left == 0) continue;
+            any = true;
+            if (round > 0 && !wait_mbar(saddr(&ctl->empty[slot]), (round - 1) & 1u, ctl, a.error_flag, 14)) return false;
+            if (poisoned(ctl)) return false;
+            const uint32_t bar = saddr(&ctl->full[slot]);
+            if (cur[w].j == cur[w].nb - 1) {
+                mbar_arrive(bar);
+            } else {
+                const int left_rows = cur[w].rows - 32 * cur[w].j;
+                const uint32_t bytes = (uint32_t)(left_rows < 32 ? left_rows : 32) * (DH * 2);
+                const int kvh = cur[w].hg * GQ / Gh;
+                const long long off =
+                    (((long long)__ldg(a.slots + cur[w].b) * a.Hkv + kvh) * (long long)a.max_len + 32 * cur[w].j) * DH;
+                mbar_expect_tx(bar, 2 * bytes);
+                const uint32_t dst = smemA + slot * TC_A_BYTES;
+                bulk_load(dst, (const bf16*)a.Kc + off, bytes, bar);
+                bulk_load(dst + 32 * DH * 2, (const bf16*)a.Vc + off, bytes, bar);
+            }
+            attw_cursor_next(cur[w], a.pos0, HG);
+            if (++slot == TC_STAGES) { slot = 0; ++round; }
+            st_release_cta_u32(&ctl->issued, round * TC_STAGES + slot);
+        }
+    }
+    return true;
+}
+
 // ---- producers -------------------------------------------------------------------------------------
 // Weight tiles: arms the stage's barrier with the bytes of both tiles and issues the weight copy.  Runs
-// ahead of the grid barriers, limited only by the ring.
-__device__ void tc_producer_w(const TcParams& P, TcCtl* ctl, uint32_t smemA, int cta, int G) {
+// ahead of the grid barriers, limited only by the ring.  Also issues the attention items of every step.
+template <int DH, int GQ>
+__device__ void tc_producer_w(const TcParams& P, TcCtl* ctl, uint32_t smemA, int cta, int G, const TcAttInfo& ai) {
     const TcArgs& a = P.a;
     const u64 pol_w = policy_evict_first();
+    AttwCursor first[TC_ATT_WARPS];
+#pragma unroll
+    for (int w = 0; w < TC_ATT_WARPS; ++w) {
+        unsigned u0, u1;
+        attw_range(ai.pl, w * G + cta, u0, u1);
+        attw_cursor_init(first[w], a.pos0, a.Hq / GQ, u0, u1);
+    }
     Cursor c{0, 0, 0, 0, 0, 0, true, false};
     cursor_enter(c, a, cta, G);
     unsigned slot = 0, round = 0;
-    while (c.live) {
+    int att_done = 0;               // steps whose attention items have been issued
+    unsigned publish = 0;           // weight items still to be announced (those that reuse attention stages)
+    bool ok = true;
+    while (c.live && ok) {
+        const int att_need = c.step + (c.p >= PH_O ? 1 : 0);
+        while (ok && att_done < att_need) {
+            ok = tc_issue_attention<DH, GQ>(a, ctl, smemA, first, slot, round);
+            ++att_done;
+            publish = TC_STAGES;
+        }
+        if (!ok) break;
         if (round > 0 && !wait_mbar(saddr(&ctl->empty[slot]), (round - 1) & 1u, ctl, a.error_flag, 3)) break;
         if (poisoned(ctl)) break;
         const uint32_t bar = saddr(&ctl->full[slot]);
@@ -294,6 +438,14 @@ __device__ void tc_producer_w(const TcParams& P, TcCtl* ctl, uint32_t smemA, int
         tma_load_2d(smemA + slot * TC_A_BYTES, &P.maps.m[TCM_W + c.p], c.kb * TC_BK, c.tile * TC_TM, bar, pol_w);
         cursor_next(c, a, cta, G);
         if (++slot == TC_STAGES) { slot = 0; ++round; }
+        if (publish) {
+            st_release_cta_u32(&ctl->issued, round * TC_STAGES + slot);
+            --publish;
+        }
+    }
+    while (ok && !poisoned(ctl) && att_done < a.k) {
+        ok = tc_issue_attention<DH, GQ>(a, ctl, smemA, first, slot, round);
+        ++att_done;
     }
     if (poisoned(ctl)) drain_after_poison();
 }
@@ -301,7 +453,7 @@ __device__ void tc_producer_w(const TcParams& P, TcCtl* ctl, uint32_t smemA, int
 // Batch-operand tiles (one thread): same k-block order; the first tile of a phase waits for the grid barrier
 // after which the operand is complete.  The embedding half of the fusion FC reads the rows that the gather
 // of this step copied out of the embedding table, and waits for that barrier.
-__device__ void tc_producer_x(const TcParams& P, TcCtl* ctl, uint32_t smemB, int cta, int G) {
+__device__ void tc_producer_x(const TcParams& P, TcCtl* ctl, uint32_t smemB, int cta, int G, unsigned att_items) {
     const TcArgs& a = P.a;
     const u64 pol_x = policy_evict_last();
     Cursor c{0, 0, 0, 0, 0, 0, true, false};
@@ -310,7 +462,10 @@ __device__ void tc_producer_x(const TcParams& P, TcCtl* ctl, uint32_t smemB, int
     const int dkb = a.d / TC_BK;
     int map_idx = TCM_X_FEAT;
     int gathered_step = -1;
+    int att_done = 0;
     while (c.live) {
+        for (const int att_need = c.step + (c.p >= PH_O ? 1 : 0); att_done < att_need; ++att_done)
+            ring_skip(slot, round, att_items);          // the attention items between the QKV and O tiles
         if (c.entered) {
             const int need = need_seq(c.step, c.p);
             if (need >= 0) {
@@ -385,23 +540,34 @@ __device__ void tc_gather(const TcParams& P, TcCtl* ctl, int s, int cta, int G, 
 }
 
 // ---- MMA issuer ----------------------------------------------------------------------------------
-__device__ void tc_mma_issuer(const TcParams& P, TcCtl* ctl, uint32_t smemA, uint32_t smemB, int cta, int G) {
+__device__ void tc_mma_issuer(const TcParams& P, TcCtl* ctl, uint32_t smemA, uint32_t smemB, int cta, int G,
+                              unsigned att_items) {
     const TcArgs& a = P.a;
     const uint32_t tmem = ctl->tmem_base;
     unsigned seg_cnt = 0, slot = 0, round = 0;
+    unsigned check = 0;         // items whose stage last held an attention item: see wait_issued
     for (int s = 0; s < a.k; ++s)
         for (int p = 0; p < PH_COUNT; ++p) {
             const PhaseShape sh = phase_shape(a, p);
             const long long lo = range_lo(sh.W, cta, G), hi = range_lo(sh.W, cta + 1, G);
             int left = (int)(hi - lo);
             int kb0 = left > 0 ? (int)(lo % sh.nkb) : 0;
+            if (p == PH_O && att_items > 0) {                       // the attention items of this step
+                ring_skip(slot, round, att_items);
+                check = TC_STAGES;
+            }
             while (left > 0) {
                 const int n = left < sh.nkb - kb0 ? left : sh.nkb - kb0;
                 const unsigned acc = seg_cnt & 1u, use = seg_cnt >> 1;
                 if (use > 0) wait_mbar(saddr(&ctl->tempty[acc]), (use - 1) & 1u, ctl, a.error_flag, 4);
                 tc_fence_after();
                 for (int j = 0; j < n; ++j) {
-                    const bool ok = wait_mbar(saddr(&ctl->full[slot]), round & 1u, ctl, a.error_flag, 5);
+                    bool ok = true;
+                    if (check) {
+                        ok = wait_issued(ctl, round * TC_STAGES + slot, a.error_flag, 16);
+                        --check;
+                    }
+                    ok = ok && wait_mbar(saddr(&ctl->full[slot]), round & 1u, ctl, a.error_flag, 5);
                     if (ok) {
                         tc_fence_after();
                         const u64 ad = tc_smem_desc(smemA + slot * TC_A_BYTES);
@@ -713,6 +879,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
             mbar_init(saddr(&ctl->tempty[i]), TC_EPI_THREADS);
         }
         ctl->abort_flag = 0;
+        ctl->issued = 0;
         ctl->wait_cycles = a.wait_cycles;
         ctl->last_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -728,14 +895,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
     __syncthreads();
     tc_fence_after();
 
+    // the split of the attention units (the same for every step) and this CTA's ring items per step
+    const TcAttInfo ai = tc_att_info(a, a.Hq / GQ, cta, G);
     if (warp == 0) {
-        if (lane == 0) tc_producer_w(P, ctl, smemA, cta, G);
+        if (lane == 0) tc_producer_w<DH, GQ>(P, ctl, smemA, cta, G, ai);
         __syncwarp();
     } else if (warp == 1) {
-        if (lane == 0) tc_mma_issuer(P, ctl, smemA, smemB, cta, G);
+        if (lane == 0) tc_mma_issuer(P, ctl, smemA, smemB, cta, G, ai.total);
         __syncwarp();
     } else if (warp == 2) {
-        if (lane == 0) tc_producer_x(P, ctl, smemB, cta, G);
+        if (lane == 0) tc_producer_x(P, ctl, smemB, cta, G, ai.total);
         __syncwarp();
     } else {
         // warps 4..7: epilogue of every GEMM phase; warp 3: the embedding gather; warps 3..7: the attention
@@ -749,6 +918,18 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
         aw.pos0 = a.pos0; aw.step = 0; aw.rope_tab = a.rope_tab; aw.Hq = a.Hq; aw.Hkv = a.Hkv; aw.max_len = a.max_len;
         aw.B = a.B; aw.scale = a.scale; aw.part_acc = a.part_acc; aw.part_ml = a.part_ml; aw.nslot = a.attn_nslot;
         aw.counters = a.counters; aw.attn = a.attn; aw.attn_h = a.attn_h; aw.lo_rows = a.lo ? a.B : 0;
+        // ring items of this CTA per step, and those before the attention items of step 0
+        unsigned items_step = ai.total, items_before = 0;
+        for (int p = 0; p < PH_COUNT; ++p) {
+            const PhaseShape sh = phase_shape(a, p);
+            const unsigned cnt = (unsigned)(range_lo(sh.W, cta + 1, G) - range_lo(sh.W, cta, G));
+            items_step += cnt;
+            if (p < PH_O) items_before += cnt;
+        }
+        TcAttRing ring;
+        ring.ctl = ctl; ring.error_flag = a.error_flag; ring.smemA = smemA; ring.w = warp - 3;
+#pragma unroll
+        for (int w = 0; w < TC_ATT_WARPS; ++w) ring.n[w] = ai.n[w];
         for (int s = 0; s < a.k; ++s) {
             if (is_epi) {
                 tc_epilogue_phase(P, ctl, s, PH_FC, seg_cnt, cta, G, w4, lane);
@@ -763,7 +944,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
             if (!poisoned(ctl)) {
                 aw.step = s;
                 aw.rope_tab = a.rope_tab + (long long)(s & 1) * 16 * (DH / 2);
-                attn_warp_phase<DH, GQ>(aw, cta * TC_ATT_WARPS + (warp - 3), G * TC_ATT_WARPS, lane);
+                ring.base = items_before + (unsigned)s * items_step;
+                attn_warp_phase<DH, GQ>(aw, ai.pl, (warp - 3) * G + cta, lane, ring);
             }
             named_sync(TC_BAR_ATT, TC_ATT_WARPS * 32);
             if (atid == 0) {
