@@ -65,7 +65,8 @@ struct TcCtl {
     unsigned issued;            // ring items the weight producer has armed so far
     int abort_flag;
     long long wait_cycles;      // limit of every wait
-    int last_flag, c_first, c_first_slot, n_contrib;
+    int last_flag, early_flag;
+    int cinfo[2][3];            // contributors of the CTA's first and last tile of the phase: first CTA, its slot bit, count
     float scale[16];
     float red[8][16];
 };
@@ -162,6 +163,11 @@ __device__ __forceinline__ u64 ld_acquire_u64(const u64* p) {
 }
 __device__ __forceinline__ void red_release_add_u64(u64* p, u64 v) {
     asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ int ld_acquire_int(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
 }
 __device__ __forceinline__ int ld_relaxed_int(const int* p) {
     int v;
@@ -726,7 +732,45 @@ __device__ void epi_output(const TcArgs& a, TcCtl* ctl, int p, int s, int tile, 
 }
 
 // ---- epilogue warps: GEMM phases -------------------------------------------------------------------
+// Sum of the partial accumulators of contributors i = from, from-1, ..., to of a shared tile, folded from the
+// right: acc = c_i + acc.  Three contributors' loads are in flight together.
+__device__ __forceinline__ void fold_partials(const TcArgs& a, float (&acc)[16], int cf, int fs, int from, int to, int etid) {
+    const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 1
+    for (int i0 = from; i0 >= to; i0 -= 3) {
+        float4 t[3][4];
+#pragma unroll
+        for (int q = 0; q < 3; ++q) {
+            const int i = i0 - q;
+            const bool on = i >= to;
+            const float4* src = (const float4*)(a.partial + (long long)((cf + (on ? i : to)) * 2 + (i == 0 ? fs : 0)) * (16 * TC_TM)) + etid * 4;
+#pragma unroll
+            for (int r = 0; r < 4; ++r) t[q][r] = on ? __ldcg(src + r) : z4;
+        }
+#pragma unroll
+        for (int q = 0; q < 3; ++q) {
+            if (i0 - q < to) break;
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                acc[4 * r] = t[q][r].x + acc[4 * r];
+                acc[4 * r + 1] = t[q][r].y + acc[4 * r + 1];
+                acc[4 * r + 2] = t[q][r].z + acc[4 * r + 2];
+                acc[4 * r + 3] = t[q][r].w + acc[4 * r + 3];
+            }
+        }
+    }
+}
+
 // Runs phase p of step s for this CTA's range and arrives on the phase's grid barrier.
+//
+// A tile that this CTA shares with others is the sum of its contributors' partial accumulators, always added
+// in the same order (from the last contributor down to the first), so the result does not depend on who
+// finishes the tile.  Usually a contributor stores its partial, counts itself on the tile's arrival counter
+// and, if it was the last, adds the others' partials to its own.  When this CTA's range is at least a tile
+// long, the other contributors of the tile at the END of its range finished that tile long ago (it was the
+// first thing they did in the phase): the counter is looked at while the MMAs of the segment still run, and if
+// everybody else has arrived their partials are summed right then; once the accumulator is ready the tile is
+// finished without the store, the fence, the atomic and the loads on the critical path.
 __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, unsigned& seg_cnt, int cta, int G,
                                   int w4, int lane) {
     const TcArgs& a = P.a;
@@ -735,24 +779,47 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
     const long long lo = range_lo(sh.W, cta, G), hi = range_lo(sh.W, cta + 1, G);
     long long idx = lo;
     bool need_scale = (p == PH_QKV || p == PH_GU);
+    const bool big = sh.W >= G;        // every CTA has work: the contributors of a tile are consecutive CTAs
     // Contributors of the (at most two) tiles this CTA shares with others, worked out while the first
     // accumulator is still being computed: first contributor, its slot bit, number of contributors.
-    int cinfo[2][3] = {{0, 0, 0}, {0, 0, 0}};
-    if (etid == 0 && lo < hi && sh.W >= G) {
+    if (etid == 0 && lo < hi && big) {
         const long long tl[2] = {lo / sh.nkb, (hi - 1) / sh.nkb};
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
             const long long t0 = tl[q] * sh.nkb;
             const int cf = owner_of(sh.W, G, t0);
-            cinfo[q][0] = cf;
-            cinfo[q][1] = t0 == range_lo(sh.W, cf, G) ? 0 : 1;
-            cinfo[q][2] = owner_of(sh.W, G, t0 + sh.nkb - 1) - cf + 1;
+            ctl->cinfo[q][0] = cf;
+            ctl->cinfo[q][1] = t0 == range_lo(sh.W, cf, G) ? 0 : 1;
+            ctl->cinfo[q][2] = owner_of(sh.W, G, t0 + sh.nkb - 1) - cf + 1;
         }
     }
+    if (lo < hi && big) named_sync(TC_BAR_EPI, TC_EPI_THREADS);
     const int tile_first = (int)(lo / sh.nkb);
     while (idx < hi) {
         const int tile = (int)(idx / sh.nkb), kb0 = (int)(idx % sh.nkb);
         const int n = (int)((hi - idx) < (long long)(sh.nkb - kb0) ? (hi - idx) : (long long)(sh.nkb - kb0));
+        const bool shared = !(kb0 == 0 && n == sh.nkb);
+        int cf = 0, fs = 0, nc = 0;
+        if (shared && big) {
+            const int q = tile == tile_first ? 0 : 1;
+            cf = ctl->cinfo[q][0]; fs = ctl->cinfo[q][1]; nc = ctl->cinfo[q][2];
+        }
+        const int me = cta - cf;            // this CTA's place among the contributors (big phases)
+        // ---- while the MMAs of the segment run: the early look at the arrival counter
+        bool early = false;
+        float others[16];
+#pragma unroll
+        for (int c = 0; c < 16; ++c) others[c] = 0.f;
+        if (shared && big && idx != lo && hi - lo >= sh.nkb) {
+            if (etid == 0) {
+                const int seen = ld_acquire_int(a.tile_ctr + tile);
+                __threadfence();
+                ctl->early_flag = seen == nc - 1;
+            }
+            named_sync(TC_BAR_EPI, TC_EPI_THREADS);
+            early = ctl->early_flag != 0;
+            if (early) fold_partials(a, others, cf, fs, nc - 1, me + 1, etid);
+        }
         const unsigned acc = seg_cnt & 1u;
         wait_mbar(saddr(&ctl->tfull[acc]), (seg_cnt >> 1) & 1u, ctl, a.error_flag, 6);
         tc_fence_after();
@@ -766,30 +833,24 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
             need_scale = false;
         }
         bool finish = true;
-        if (!(kb0 == 0 && n == sh.nkb)) {
-            // a tile shared with other CTAs: publish the partial accumulator ([row][16 columns], 64 bytes per
-            // thread); the last arriver finishes the tile
+        if (shared && early) {
+#pragma unroll
+            for (int c = 0; c < 16; ++c) v[c] += others[c];
+            fold_partials(a, v, cf, fs, me - 1, 0, etid);
+            if (etid == 0) a.tile_ctr[tile] = 0;        // nobody else will come: ready for the tile's next use
+        } else if (shared) {
+            // publish the partial accumulator ([row][16 columns], 64 bytes per thread); the last arriver
+            // finishes the tile
             float4* mine = (float4*)(a.partial + (long long)(cta * 2 + (idx == lo ? 0 : 1)) * (16 * TC_TM)) + etid * 4;
 #pragma unroll
             for (int q = 0; q < 4; ++q) __stcg(mine + q, make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]));
             named_sync(TC_BAR_EPI, TC_EPI_THREADS);
             if (etid == 0) {
-                // contributors = the CTAs whose (non-empty) ranges meet this tile, in range order; when every
-                // CTA has work in the phase they are consecutive CTAs
-                int cf, fs, nc;
-                if (sh.W >= G) {
-                    const int q = tile == tile_first ? 0 : 1;
-                    cf = cinfo[q][0]; fs = cinfo[q][1]; nc = cinfo[q][2];
-                } else {
+                if (!big) {
+                    // contributors = the CTAs whose (non-empty) ranges meet this tile, in range order
                     const long long t0 = (long long)tile * sh.nkb;
-                    cf = owner_of(sh.W, G, t0);
-                    fs = t0 == range_lo(sh.W, cf, G) ? 0 : 1;
-                    nc = 0;
                     for (long long i = t0; i < t0 + sh.nkb; ++nc) i = range_lo(sh.W, owner_of(sh.W, G, i) + 1, G);
                 }
-                ctl->c_first = cf;
-                ctl->c_first_slot = fs;
-                ctl->n_contrib = nc;
                 __threadfence();                       // the CTA's partial (ordered before by the barrier) is visible first
                 const int old = atomicAdd(a.tile_ctr + tile, 1);
                 const int last = old == nc - 1;
@@ -802,28 +863,15 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
             named_sync(TC_BAR_EPI, TC_EPI_THREADS);
             finish = ctl->last_flag != 0;
             if (finish) {
-                // contributor order is fixed, so the sum does not depend on who arrived last
+                if (big) {
+                    fold_partials(a, others, cf, fs, nc - 1, me + 1, etid);
 #pragma unroll
-                for (int c = 0; c < 16; ++c) v[c] = 0.f;
-                if (sh.W >= G) {
-                    const int cf = ctl->c_first, nc = ctl->n_contrib, fs = ctl->c_first_slot;
-                    const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 1
-                    for (int j0 = 0; j0 < nc; j0 += 2) {        // loads of two contributors in flight together
-                        const float4* sa = (const float4*)(a.partial + (long long)((cf + j0) * 2 + (j0 == 0 ? fs : 0)) * (16 * TC_TM)) + etid * 4;
-                        const float4* sb = (const float4*)(a.partial + (long long)((cf + j0 + 1) * 2) * (16 * TC_TM)) + etid * 4;
-                        const bool two = j0 + 1 < nc;
-                        const float4 a0 = __ldcg(sa), a1 = __ldcg(sa + 1), a2 = __ldcg(sa + 2), a3 = __ldcg(sa + 3);
-                        const float4 b0 = two ? __ldcg(sb) : z4, b1 = two ? __ldcg(sb + 1) : z4;
-                        const float4 b2 = two ? __ldcg(sb + 2) : z4, b3 = two ? __ldcg(sb + 3) : z4;
-                        v[0] += a0.x; v[1] += a0.y; v[2] += a0.z; v[3] += a0.w; v[4] += a1.x; v[5] += a1.y; v[6] += a1.z; v[7] += a1.w;
-                        v[8] += a2.x; v[9] += a2.y; v[10] += a2.z; v[11] += a2.w; v[12] += a3.x; v[13] += a3.y; v[14] += a3.z; v[15] += a3.w;
-                        if (two) {
-                            v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
-                            v[8] += b2.x; v[9] += b2.y; v[10] += b2.z; v[11] += b2.w; v[12] += b3.x; v[13] += b3.y; v[14] += b3.z; v[15] += b3.w;
-                        }
-                    }
+                    for (int c = 0; c < 16; ++c) v[c] += others[c];
+                    fold_partials(a, v, cf, fs, me - 1, 0, etid);
                 } else {
+                    // few tile-k-blocks (tiny shapes): contributors in range order, all read back
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) v[c] = 0.f;
                     const long long t0 = (long long)tile * sh.nkb;
                     for (long long i = t0; i < t0 + sh.nkb;) {
                         const int cc = owner_of(sh.W, G, i);
