@@ -69,6 +69,7 @@ struct TcCtl {
     int cinfo[2][3];            // contributors of the CTA's first and last tile of the phase: first CTA, its slot bit, count
     float scale[16];
     float red[8][16];
+    u64 kred[2][4][16];         // LM head: best key of each epilogue warp per sequence (two buffers, used in turn)
 };
 
 __device__ __forceinline__ uint32_t saddr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -640,7 +641,43 @@ __device__ __forceinline__ void epi_compute_scales(const TcArgs& a, TcCtl* ctl, 
     named_sync(TC_BAR_EPI, TC_EPI_THREADS);
 }
 
-__device__ void epi_output(const TcArgs& a, TcCtl* ctl, int p, int s, int tile, const float (&v)[16], int w4, int lane) {
+// What the output stage of a tile adds to or multiplies with the accumulators: requested before the tile's
+// accumulator is waited for, so that these round trips to L2 are over when it arrives.  Everything read here
+// was complete before the phase began (residual rows and gains are constants; u is written by the FC phase and
+// read in the O phase, y by the O phase and read in the down phase).
+struct EpiPre {
+    float add[16];      // per sequence: the residual stream the result is added to (FC: the step's residual row)
+    float g;            // RMSNorm gain of the row (FC, O) or the QKV bias
+};
+__device__ __forceinline__ void epi_preload(const TcArgs& a, int p, int s, int tile, int w4, int lane, EpiPre& pre) {
+    const int N = a.ph[p].N;
+    const int row = tile * TC_TM + w4 * 32 + lane;
+    const bool rok = row < N;
+    pre.g = 0.f;
+#pragma unroll
+    for (int b = 0; b < 16; ++b) pre.add[b] = 0.f;
+    if (!rok) return;
+    if (p == PH_FC) {
+        pre.g = __bfloat162float(a.norm1[row]);
+        const float add0 = a.rho ? a.rho[(long long)(s < a.n_resid - 1 ? s : a.n_resid - 1) * a.d + row] : 0.f;
+#pragma unroll
+        for (int b = 0; b < 16; ++b) pre.add[b] = add0;
+    } else if (p == PH_O) {
+        pre.g = __bfloat162float(a.norm2[row]);
+#pragma unroll
+        for (int b = 0; b < 16; ++b)
+            if (b < a.B) pre.add[b] = __ldcg(a.u + (long long)b * N + row);
+    } else if (p == PH_DOWN) {
+#pragma unroll
+        for (int b = 0; b < 16; ++b)
+            if (b < a.B) pre.add[b] = __ldcg(a.y + (long long)b * N + row);
+    } else if (p == PH_QKV) {
+        pre.g = a.bqkv ? __bfloat162float(a.bqkv[row]) : 0.f;
+    }
+}
+
+__device__ void epi_output(const TcArgs& a, TcCtl* ctl, int p, int s, int tile, const float (&v)[16], const EpiPre& pre,
+                           unsigned& lm_calls, int w4, int lane) {
     const int N = a.ph[p].N;
     const int row = tile * TC_TM + w4 * 32 + lane;
     const bool rok = row < N;
@@ -654,25 +691,17 @@ __device__ void epi_output(const TcArgs& a, TcCtl* ctl, int p, int s, int tile, 
         if (b < B) val[b] = v[b] + ((a.lo && b + B < 16) ? v[(b + B) & 15] : 0.f);
 
     if (p == PH_FC || p == PH_O) {
-        const float* rho = (p == PH_FC && a.rho) ? a.rho + (long long)(s < a.n_resid - 1 ? s : a.n_resid - 1) * a.d : nullptr;
-        const bf16* gamma = p == PH_FC ? a.norm1 : a.norm2;
         float* outf = p == PH_FC ? a.u : a.y;
         bf16* outh = p == PH_FC ? a.xq_h : a.xm_h;
         float* ssq = p == PH_FC ? a.ssq1 : a.ssq2;
-        const float g = rok ? __bfloat162float(gamma[row]) : 0.f;
-        const float add0 = (rok && rho) ? rho[row] : 0.f;
-        // the addends of all sequences are requested before any store (stores would order the loads behind them)
-        float add[16];
-#pragma unroll
-        for (int b = 0; b < 16; ++b) add[b] = (p == PH_O && rok && b < B) ? __ldcg(a.u + (long long)b * N + row) : add0;
         float sq[16];
 #pragma unroll
         for (int b = 0; b < 16; ++b) {
             float r = 0.f;
             if (rok && b < B) {
-                r = val[b] + add[b];
+                r = val[b] + pre.add[b];
                 outf[(long long)b * N + row] = r;
-                store_operand(outh, N, b, row, g * r, lo_rows);
+                store_operand(outh, N, b, row, pre.g * r, lo_rows);
             }
             sq[b] = r * r;
         }
@@ -680,37 +709,34 @@ __device__ void epi_output(const TcArgs& a, TcCtl* ctl, int p, int s, int tile, 
         const int col = warp_col16(lane);
         if ((lane & 1) == 0 && col < B) ssq[(long long)(tile * 4 + w4) * 16 + col] = tot;
     } else if (p == PH_QKV) {
-        const float bias = (rok && a.bqkv) ? __bfloat162float(a.bqkv[row]) : 0.f;
         if (rok) {
 #pragma unroll
             for (int b = 0; b < 16; ++b) {
                 if (b >= B) break;
-                a.qkv[(long long)b * N + row] = val[b] * ctl->scale[b] + bias;
+                a.qkv[(long long)b * N + row] = val[b] * ctl->scale[b] + pre.g;
             }
         }
     } else if (p == PH_GU) {
-        // even rows are gate_i, odd rows up_i (i = row / 2): adjacent lanes exchange their values
+        // Even rows are gate_i, odd rows up_i (i = row / 2).  Of every pair of sequences (2q, 2q + 1) the even
+        // lane finishes 2q and the odd lane 2q + 1: each sends the neighbour the value the neighbour needs and
+        // computes one SiLU(gate) * up per pair, without a branch, so that the eight of them overlap.
         const int F = N >> 1;
+        const bool odd = (lane & 1) != 0;
 #pragma unroll
-        for (int b = 0; b < 16; ++b) {
-            if (b >= B) break;
-            const float mine = val[b] * ctl->scale[b];
-            const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
-            if (rok && ((b & 1) == (lane & 1))) {
-                const float gate = (lane & 1) ? other : mine, up = (lane & 1) ? mine : other;
-                const float act = gate / (1.f + expf(-gate)) * up;
-                store_operand(a.act_h, F, b, row >> 1, act, lo_rows);
-            }
+        for (int q = 0; q < 8; ++q) {
+            const float m0 = val[2 * q] * ctl->scale[2 * q], m1 = val[2 * q + 1] * ctl->scale[2 * q + 1];
+            const float recv = __shfl_xor_sync(0xffffffffu, odd ? m0 : m1, 1);
+            const float gate = odd ? recv : m0, up = odd ? m1 : recv;
+            const float act = __fdividef(gate, 1.f + __expf(-gate)) * up;
+            const int b = 2 * q + (odd ? 1 : 0);
+            if (rok && b < B) store_operand(a.act_h, F, b, row >> 1, act, lo_rows);
         }
     } else if (p == PH_DOWN) {
         if (rok) {
-            float add[16];
-#pragma unroll
-            for (int b = 0; b < 16; ++b) add[b] = b < B ? __ldcg(a.y + (long long)b * N + row) : 0.f;
 #pragma unroll
             for (int b = 0; b < 16; ++b) {
                 if (b >= B) break;
-                const float r = add[b] + val[b];
+                const float r = pre.add[b] + val[b];
                 a.feat[(long long)b * N + row] = r;
                 store_operand(a.feat_h, N, b, row, r, lo_rows);
             }
@@ -725,9 +751,21 @@ __device__ void epi_output(const TcArgs& a, TcCtl* ctl, int p, int s, int tile, 
                 keys[b] = pack_key(val[b], row);
             }
         }
+        // best key per sequence: over the warp, then over the four warps through shared memory, so that one
+        // atomic per sequence and tile reaches the (much contended) global keys
         const u64 best = warp_reduce16(keys, lane, OpMaxU64());
         const int col = warp_col16(lane);
-        if ((lane & 1) == 0 && col < B && best) atomicMax(a.keys + (long long)col * a.key_stride + s, best);
+        u64 (*kred)[16] = ctl->kred[lm_calls & 1u];
+        ++lm_calls;
+        if ((lane & 1) == 0) kred[w4][col] = best;
+        named_sync(TC_BAR_EPI, TC_EPI_THREADS);
+        const int etid = w4 * 32 + lane;
+        if (etid < B) {
+            u64 m = kred[0][etid];
+#pragma unroll
+            for (int w = 1; w < 4; ++w) m = kred[w][etid] > m ? kred[w][etid] : m;
+            if (m) atomicMax(a.keys + (long long)etid * a.key_stride + s, m);
+        }
     }
 }
 
@@ -778,6 +816,7 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
     const PhaseShape sh = phase_shape(a, p);
     const long long lo = range_lo(sh.W, cta, G), hi = range_lo(sh.W, cta + 1, G);
     long long idx = lo;
+    unsigned lm_calls = 0;
     bool need_scale = (p == PH_QKV || p == PH_GU);
     const bool big = sh.W >= G;        // every CTA has work: the contributors of a tile are consecutive CTAs
     // Contributors of the (at most two) tiles this CTA shares with others, worked out while the first
@@ -805,6 +844,8 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
             cf = ctl->cinfo[q][0]; fs = ctl->cinfo[q][1]; nc = ctl->cinfo[q][2];
         }
         const int me = cta - cf;            // this CTA's place among the contributors (big phases)
+        EpiPre pre;
+        epi_preload(a, p, s, tile, w4, lane, pre);
         // ---- while the MMAs of the segment run: the early look at the arrival counter
         bool early = false;
         float others[16];
@@ -887,7 +928,7 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
             }
             named_sync(TC_BAR_EPI, TC_EPI_THREADS);      // last_flag may be rewritten by the next segment
         }
-        if (finish) epi_output(a, ctl, p, s, tile, v, w4, lane);
+        if (finish) epi_output(a, ctl, p, s, tile, v, pre, lm_calls, w4, lane);
         idx += n;
     }
     // This CTA's part of the phase is done: arrive on the grid barrier.  All arrivals are counted in one
@@ -902,6 +943,9 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
         fence_proxy_async_all();
         red_release_add_u64(a.bar_counter, 1ull);
     }
+    // Without work in the phase nothing but the wait above tells this CTA that the earlier phases are complete:
+    // hold the other epilogue threads until it is over (they read those phases' results early in the next one).
+    if (lo == hi) named_sync(TC_BAR_EPI, TC_EPI_THREADS);
 }
 
 }  // namespace
