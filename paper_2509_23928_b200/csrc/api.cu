@@ -366,7 +366,8 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
         if (ok2) ok2 = cudaMemsetAsync(c->tile_ctr, 0, c->tc_tiles * sizeof(int), st) == cudaSuccess;
         if (ok2)
             ok2 = tc_build_maps(&c->tc_maps, ca.ph, cfg->d, c->qw, cfg->ffn, c->feat_h, c->xq, c->attn_h, c->xm, c->act_h,
-                                c->xe_h) == cudaSuccess;
+                                c->xe_h, c->Kc, c->Vc, MB * (long long)cfg->n_kv_heads * cfg->max_len,
+                                cfg->head_dim) == cudaSuccess;
         if (!ok2) cudaGetLastError();
         c->tc_ok = ok2;
     }

@@ -145,6 +145,7 @@ struct CuSeqlens {
 enum { TCM_W = 0,              // PH_COUNT weight maps, box 64 x 128
        TCM_X_FEAT = PH_COUNT, TCM_X_XQ, TCM_X_ATTN, TCM_X_XM, TCM_X_ACT,   // operand maps, box 64 x 16
        TCM_X_EMB,              // gathered embedding rows, box 64 x 16
+       TCM_K, TCM_V,           // the caches, box 64 x 32 rows
        TCM_COUNT };
 struct TcMaps {
     alignas(64) unsigned char m[TCM_COUNT][128];     // CUtensorMap objects
@@ -183,7 +184,8 @@ struct TcArgs {
 };
 // fills `maps` for the given buffers; returns cudaSuccess or an error (driver entry point missing, bad shape)
 cudaError_t tc_build_maps(TcMaps* maps, const ChainPhase* ph, int d, int qw, int F, const bf16* feat_h,
-                          const bf16* xq_h, const bf16* attn_h, const bf16* xm_h, const bf16* act_h, const bf16* xe_h);
+                          const bf16* xq_h, const bf16* attn_h, const bf16* xm_h, const bf16* act_h, const bf16* xe_h,
+                          const void* Kc, const void* Vc, long long cache_rows, int dh);
 bool tc_supported(int d, int dh, int Hq, int Hkv, int F);
 int tc_max_tiles(const ChainPhase* ph);
 cudaError_t launch_tc_chain(const TcMaps& maps, const TcArgs& a, int grid, cudaStream_t st);

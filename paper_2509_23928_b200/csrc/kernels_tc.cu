@@ -34,7 +34,9 @@
 // barriers still pair up, tensor memory is freed and the kernel returns.
 #include <cuda.h>
 
-#include "attn_warp.cuh"
+#include <type_traits>
+
+#include "attn_mma.cuh"
 
 #define TC_THREADS 256
 #define TC_STAGES 12
@@ -201,13 +203,16 @@ __device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, TcCtl* 
 // the parity of its phase, so whoever does not consume the ring strictly in order (the attention warps; the
 // MMA issuer after it stepped over attention items) first makes sure the stage is in the phase it means to
 // wait for: the producer arms item idx only after item idx - TC_STAGES has been handed back.
+// The count is a plain shared-memory word written after the arming by the same thread: operations of one
+// thread on the CTA's shared memory (the barrier's arrive included) take effect in program order, so a reader
+// that sees the count finds the barrier armed.  (A release/acquire pair here costs a fence per ring item.)
 __device__ __forceinline__ unsigned ld_acquire_cta_u32(const unsigned* p) {
     unsigned v;
-    asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(saddr(p)) : "memory");
+    asm volatile("ld.volatile.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(saddr(p)) : "memory");
     return v;
 }
 __device__ __forceinline__ void st_release_cta_u32(unsigned* p, unsigned v) {
-    asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(saddr(p)), "r"(v) : "memory");
+    asm volatile("st.volatile.shared::cta.u32 [%0], %1;" ::"r"(saddr(p)), "r"(v) : "memory");
 }
 __device__ __forceinline__ bool wait_issued(TcCtl* ctl, unsigned idx, int* error_flag, int code) {
     if (poisoned(ctl)) return false;
@@ -322,20 +327,39 @@ __device__ __forceinline__ void drain_after_poison() {
 // QKV tiles and the O tiles of the step the weight producer issues one item per attention unit of this CTA's
 // attention warps, round-robin over the warps (round r: the r-th unit of every warp that has one).  The
 // attention warps consume these items; the MMA issuer and the operand producer step over them.
+// Two attention bodies share this machinery: groups of query heads on one KV head (GQ > 1) take the tensor-core
+// body (attn_mma.cuh: one key or part of a key per warp, swizzled stages), single heads the FMA body
+// (attn_warp.cuh: equal unit ranges per warp, plain stages).
+template <int GQ> struct AttSel { static constexpr bool mma = GQ > 1; };
 struct TcAttInfo {
-    AttwPlan pl;
+    AttwPlan pl;                    // FMA body: the split of the unit list
+    AttmPlan plm;                   // tensor-core body: the plan and the work of each attention warp of this CTA
+    AttmJob job[TC_ATT_WARPS];
     unsigned n[TC_ATT_WARPS];       // units of attention warp w of this CTA (global warp number w * G + cta)
     unsigned total;
 };
-__device__ __forceinline__ TcAttInfo tc_att_info(const TcArgs& a, int HG, int cta, int G) {
+template <int GQ>
+__device__ __forceinline__ TcAttInfo tc_att_info(const TcArgs& a, int cta, int G) {
+    const int HG = a.Hq / GQ;
     TcAttInfo t;
-    t.pl = attw_plan(a.pos0, a.B, HG, G * TC_ATT_WARPS);
     t.total = 0;
+    if constexpr (AttSel<GQ>::mma) {
+        t.plm = attm_plan(a.pos0, a.B, HG, G * TC_ATT_WARPS);
+        t.pl.U = 0; t.pl.NW = 0;
+    } else {
+        t.pl = attw_plan(a.pos0, a.B, HG, G * TC_ATT_WARPS);
+        t.plm.T = 0; t.plm.NW = 0; t.plm.nkeys = 0;
+    }
 #pragma unroll
     for (int w = 0; w < TC_ATT_WARPS; ++w) {
-        unsigned u0, u1;
-        attw_range(t.pl, w * G + cta, u0, u1);
-        t.n[w] = u1 - u0;
+        if constexpr (AttSel<GQ>::mma) {
+            t.job[w] = attm_job(t.plm, a.pos0, a.B, HG, w * G + cta);
+            t.n[w] = t.job[w].units;
+        } else {
+            unsigned u0, u1;
+            attw_range(t.pl, w * G + cta, u0, u1);
+            t.n[w] = u1 - u0;
+        }
         t.total += t.n[w];
     }
     return t;
@@ -369,13 +393,19 @@ struct TcAttRing {
     __device__ __forceinline__ void release(unsigned r) { mbar_arrive(saddr(&ctl->empty[position(r) % TC_STAGES])); }
 };
 
-// One step's attention items (producer thread).  A prefix block is two bulk copies: its K rows to the start
-// of the stage, its V rows behind the room of 32 K rows.  The prefix is not written during the launch, so
-// these copies need no grid barrier.  A tail unit is an item without data.
+// One step's attention items (producer thread).  The prefix is not written during the launch, so these copies
+// need no grid barrier.  A tail unit is an item without data.  A prefix block is
+//   FMA body:         two bulk copies, its K rows to the start of the stage, its V rows behind the room of 32 K
+//                     rows;
+//   tensor-core body: a tiled copy per 64 elements of the head dimension, of 32 cache rows each, for K and for V
+//                     (128-byte swizzle, which the matrix loads want); rows of the box beyond the prefix are
+//                     fetched too and never used.
+template <int GQ> using AttCursor = std::conditional_t<AttSel<GQ>::mma, AttmCursor, AttwCursor>;
 template <int DH, int GQ>
-__device__ bool tc_issue_attention(const TcArgs& a, TcCtl* ctl, uint32_t smemA, const AttwCursor (&first)[TC_ATT_WARPS],
-                                   unsigned& slot, unsigned& round) {
-    AttwCursor cur[TC_ATT_WARPS];
+__device__ bool tc_issue_attention(const TcParams& P, TcCtl* ctl, uint32_t smemA, const AttCursor<GQ> (&first)[TC_ATT_WARPS],
+                                   unsigned& slot, unsigned& round, u64 pol) {
+    const TcArgs& a = P.a;
+    AttCursor<GQ> cur[TC_ATT_WARPS];
 #pragma unroll
     for (int w = 0; w < TC_ATT_WARPS; ++w) cur[w] = first[w];
     const int HG = a.Hq / GQ, Gh = a.Hq / a.Hkv;
@@ -392,17 +422,28 @@ __device__ bool tc_issue_attention(const TcArgs& a, TcCtl* ctl, uint32_t smemA, 
             if (cur[w].j == cur[w].nb - 1) {
                 mbar_arrive(bar);
             } else {
-                const int left_rows = cur[w].rows - 32 * cur[w].j;
-                const uint32_t bytes = (uint32_t)(left_rows < 32 ? left_rows : 32) * (DH * 2);
                 const int kvh = cur[w].hg * GQ / Gh;
-                const long long off =
-                    (((long long)__ldg(a.slots + cur[w].b) * a.Hkv + kvh) * (long long)a.max_len + 32 * cur[w].j) * DH;
-                mbar_expect_tx(bar, 2 * bytes);
                 const uint32_t dst = smemA + slot * TC_A_BYTES;
-                bulk_load(dst, (const bf16*)a.Kc + off, bytes, bar);
-                bulk_load(dst + 32 * DH * 2, (const bf16*)a.Vc + off, bytes, bar);
+                if constexpr (AttSel<GQ>::mma) {
+                    const int row0 = (cur[w].slot * a.Hkv + kvh) * a.max_len + 32 * cur[w].j;
+                    mbar_expect_tx(bar, 2 * 32 * DH * 2);
+#pragma unroll
+                    for (int h = 0; h < DH / 64; ++h) {
+                        tma_load_2d(dst + h * 4096, &P.maps.m[TCM_K], 64 * h, row0, bar, pol);
+                        tma_load_2d(dst + 32 * DH * 2 + h * 4096, &P.maps.m[TCM_V], 64 * h, row0, bar, pol);
+                    }
+                } else {
+                    const int left_rows = cur[w].rows - 32 * cur[w].j;
+                    const uint32_t bytes = (uint32_t)(left_rows < 32 ? left_rows : 32) * (DH * 2);
+                    const long long off =
+                        (((long long)__ldg(a.slots + cur[w].b) * a.Hkv + kvh) * (long long)a.max_len + 32 * cur[w].j) * DH;
+                    mbar_expect_tx(bar, 2 * bytes);
+                    bulk_load(dst, (const bf16*)a.Kc + off, bytes, bar);
+                    bulk_load(dst + 32 * DH * 2, (const bf16*)a.Vc + off, bytes, bar);
+                }
             }
-            attw_cursor_next(cur[w], a.pos0, HG);
+            if constexpr (AttSel<GQ>::mma) attm_cursor_next(cur[w], a.pos0, a.slots, HG);
+            else attw_cursor_next(cur[w], a.pos0, HG);
             if (++slot == TC_STAGES) { slot = 0; ++round; }
             st_release_cta_u32(&ctl->issued, round * TC_STAGES + slot);
         }
@@ -417,12 +458,17 @@ template <int DH, int GQ>
 __device__ void tc_producer_w(const TcParams& P, TcCtl* ctl, uint32_t smemA, int cta, int G, const TcAttInfo& ai) {
     const TcArgs& a = P.a;
     const u64 pol_w = policy_evict_first();
-    AttwCursor first[TC_ATT_WARPS];
+    const u64 pol_kv = policy_evict_last();       // the cache is read again at every step
+    AttCursor<GQ> first[TC_ATT_WARPS];
 #pragma unroll
     for (int w = 0; w < TC_ATT_WARPS; ++w) {
-        unsigned u0, u1;
-        attw_range(ai.pl, w * G + cta, u0, u1);
-        attw_cursor_init(first[w], a.pos0, a.Hq / GQ, u0, u1);
+        if constexpr (AttSel<GQ>::mma) {
+            attm_cursor_init(first[w], ai.job[w], a.pos0, a.slots, a.Hq / GQ);
+        } else {
+            unsigned u0, u1;
+            attw_range(ai.pl, w * G + cta, u0, u1);
+            attw_cursor_init(first[w], a.pos0, a.Hq / GQ, u0, u1);
+        }
     }
     Cursor c{0, 0, 0, 0, 0, 0, true, false};
     cursor_enter(c, a, cta, G);
@@ -433,7 +479,7 @@ __device__ void tc_producer_w(const TcParams& P, TcCtl* ctl, uint32_t smemA, int
     while (c.live && ok) {
         const int att_need = c.step + (c.p >= PH_O ? 1 : 0);
         while (ok && att_done < att_need) {
-            ok = tc_issue_attention<DH, GQ>(a, ctl, smemA, first, slot, round);
+            ok = tc_issue_attention<DH, GQ>(P, ctl, smemA, first, slot, round, pol_kv);
             ++att_done;
             publish = TC_STAGES;
         }
@@ -451,7 +497,7 @@ __device__ void tc_producer_w(const TcParams& P, TcCtl* ctl, uint32_t smemA, int
         }
     }
     while (ok && !poisoned(ctl) && att_done < a.k) {
-        ok = tc_issue_attention<DH, GQ>(a, ctl, smemA, first, slot, round);
+        ok = tc_issue_attention<DH, GQ>(P, ctl, smemA, first, slot, round, pol_kv);
         ++att_done;
     }
     if (poisoned(ctl)) drain_after_poison();
@@ -771,14 +817,16 @@ __device__ void epi_output(const TcArgs& a, TcCtl* ctl, int p, int s, int tile, 
 
 // ---- epilogue warps: GEMM phases -------------------------------------------------------------------
 // Sum of the partial accumulators of contributors i = from, from-1, ..., to of a shared tile, folded from the
-// right: acc = c_i + acc.  Three contributors' loads are in flight together.
+// right: acc = c_i + acc.  Up to TC_FOLD contributors' loads are in flight together (the phases with few row
+// tiles have five or six contributors per tile, all finishing at the same moment: one round trip, not three).
+#define TC_FOLD 5
 __device__ __forceinline__ void fold_partials(const TcArgs& a, float (&acc)[16], int cf, int fs, int from, int to, int etid) {
     const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 1
-    for (int i0 = from; i0 >= to; i0 -= 3) {
-        float4 t[3][4];
+    for (int i0 = from; i0 >= to; i0 -= TC_FOLD) {
+        float4 t[TC_FOLD][4];
 #pragma unroll
-        for (int q = 0; q < 3; ++q) {
+        for (int q = 0; q < TC_FOLD; ++q) {
             const int i = i0 - q;
             const bool on = i >= to;
             const float4* src = (const float4*)(a.partial + (long long)((cf + (on ? i : to)) * 2 + (i == 0 ? fs : 0)) * (16 * TC_TM)) + etid * 4;
@@ -786,7 +834,7 @@ __device__ __forceinline__ void fold_partials(const TcArgs& a, float (&acc)[16],
             for (int r = 0; r < 4; ++r) t[q][r] = on ? __ldcg(src + r) : z4;
         }
 #pragma unroll
-        for (int q = 0; q < 3; ++q) {
+        for (int q = 0; q < TC_FOLD; ++q) {
             if (i0 - q < to) break;
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
@@ -988,7 +1036,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
     tc_fence_after();
 
     // the split of the attention units (the same for every step) and this CTA's ring items per step
-    const TcAttInfo ai = tc_att_info(a, a.Hq / GQ, cta, G);
+    const TcAttInfo ai = tc_att_info<GQ>(a, cta, G);
     if (warp == 0) {
         if (lane == 0) tc_producer_w<DH, GQ>(P, ctl, smemA, cta, G, ai);
         __syncwarp();
@@ -1037,7 +1085,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
                 aw.step = s;
                 aw.rope_tab = a.rope_tab + (long long)(s & 1) * 16 * (DH / 2);
                 ring.base = items_before + (unsigned)s * items_step;
-                attn_warp_phase<DH, GQ>(aw, ai.pl, (warp - 3) * G + cta, lane, ring);
+                if constexpr (AttSel<GQ>::mma) attn_mma_phase<DH, GQ>(aw, ai.job[warp - 3], lane, ring);
+                else attn_warp_phase<DH, GQ>(aw, ai.pl, (warp - 3) * G + cta, lane, ring);
             }
             named_sync(TC_BAR_ATT, TC_ATT_WARPS * 32);
             if (atid == 0) {
@@ -1147,7 +1196,7 @@ int tc_barriers_per_step() { return TC_BARS_PER_STEP; }
 
 cudaError_t tc_build_maps(TcMaps* maps, const ChainPhase* ph, int d, int qw, int F,
                           const bf16* feat_h, const bf16* xq_h, const bf16* attn_h, const bf16* xm_h,
-                          const bf16* act_h, const bf16* xe_h) {
+                          const bf16* act_h, const bf16* xe_h, const void* Kc, const void* Vc, long long cache_rows, int dh) {
     static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
     cudaError_t e;
     for (int p = 0; p < PH_COUNT; ++p) {
@@ -1160,7 +1209,12 @@ cudaError_t tc_build_maps(TcMaps* maps, const ChainPhase* ph, int d, int qw, int
         e = encode_map(maps->m[ops[i].idx], ops[i].base, TC_OP_ROWS, ops[i].cols, TC_TN, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
         if (e != cudaSuccess) return e;
     }
-    return encode_map(maps->m[TCM_X_EMB], xe_h, TC_OP_ROWS, d, TC_TN, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+    e = encode_map(maps->m[TCM_X_EMB], xe_h, TC_OP_ROWS, d, TC_TN, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+    if (e != cudaSuccess) return e;
+    // the caches as matrices of [slot x KV head x position] rows: boxes of 32 rows x 64 elements
+    e = encode_map(maps->m[TCM_K], Kc, cache_rows, dh, 32, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+    if (e != cudaSuccess) return e;
+    return encode_map(maps->m[TCM_V], Vc, cache_rows, dh, 32, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
 }
 
 template <int DH, int GQ>
