@@ -16,7 +16,10 @@
 //   warps 4-7            epilogue: tcgen05.ld (one weight row per thread, 16 batch values), then the fused
 //                        output stage of the phase (residuals, RMSNorm statistics and gains, RoPE-free
 //                        QKV bias, SiLU*up, LM-head argmax keys) and the bf16 operand of the next phase.
-//   warps 3-7            between the QKV and O phases: split-KV attention over the text-only cache.
+//   warps 3-7            between the QKV and O phases: split-KV attention over the text-only cache.  Its K/V
+//                        blocks travel through the same ring: the rows a sequence had when the launch began
+//                        do not change, so warp 0 copies them (between the QKV and the O tiles) ahead of the
+//                        grid barrier, and the attention warps compute from shared memory.
 //
 // Work split: a phase with T row tiles and KB k-blocks is T*KB tile-k-blocks, laid out tile-major and cut
 // into equal contiguous ranges, one per CTA (so every SM streams the same number of bytes whatever the
