@@ -130,6 +130,9 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
+__device__ __forceinline__ void prefetch_tensormap(const void* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -524,13 +527,15 @@ __device__ void tc_producer_x(const TcParams& P, TcCtl* ctl, uint32_t smemB, int
             ring_skip(slot, round, att_items);          // the attention items between the QKV and O tiles
         if (c.entered) {
             const int need = need_seq(c.step, c.p);
+            map_idx = c.p == PH_QKV ? TCM_X_XQ : c.p == PH_O ? TCM_X_ATTN : c.p == PH_GU ? TCM_X_XM
+                    : c.p == PH_DOWN ? TCM_X_ACT : TCM_X_FEAT;
+            // the descriptor of the phase's operand is asked for while the barrier is still awaited
+            prefetch_tensormap(&P.maps.m[map_idx]);
             if (need >= 0) {
                 if (!wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(need + 1), ctl, a.error_flag, 9)) break;
                 // other CTAs wrote the operand through the generic proxy; TMA reads through the async proxy
                 fence_proxy_async_all();
             }
-            map_idx = c.p == PH_QKV ? TCM_X_XQ : c.p == PH_O ? TCM_X_ATTN : c.p == PH_GU ? TCM_X_XM
-                    : c.p == PH_DOWN ? TCM_X_ACT : TCM_X_FEAT;
         }
         const bool emb = c.p == PH_FC && c.kb >= dkb;
         if (emb && gathered_step != c.step) {
