@@ -111,6 +111,12 @@ MINI_MHA = DrafterDims(d=512, n_q_heads=4, n_kv_heads=4, head_dim=128, ffn=1376,
 MINI_GQA = DrafterDims(d=448, n_q_heads=7, n_kv_heads=1, head_dim=64, ffn=1184, vocab=5031,
                        rms_eps=1e-6, dtype="bf16")
 
+# Many heads at a small width: more (sequence, head group) pairs than a B200 has attention warps (740).
+WIDE_GQA = DrafterDims(d=128, n_q_heads=336, n_kv_heads=48, head_dim=64, ffn=256, vocab=1000,
+                       rms_eps=1e-6, dtype="bf16")
+WIDE_MHA = DrafterDims(d=128, n_q_heads=48, n_kv_heads=48, head_dim=64, ffn=256, vocab=1000,
+                       rms_eps=1e-5, dtype="bf16")
+
 WORKLOADS: Dict[str, Workload] = {w.name: w for w in [
     Workload("c1_tiny_f32_b1", TINY, batch=1, k=4, seed=1001, text_len=32, logits_dtype="f32"),
     Workload("c2_llava_b1", LLAVA, batch=1, k=5, seed=1002, text_len=128, logits_dtype="bf16"),
@@ -130,6 +136,10 @@ WORKLOADS: Dict[str, Workload] = {w.name: w for w in [
     Workload("mini_gqa_b3", MINI_GQA, batch=3, k=2, seed=2004, text_len=65, logits_dtype="bf16"),
     Workload("tiny_f32_b4_ragged", TINY, batch=4, k=6, seed=2005, text_len_range=(1, 70),
              logits_dtype="f32"),
+    Workload("wide_gqa_b16_ragged", WIDE_GQA, batch=16, k=3, seed=2006, text_len_range=(2, 70),
+             logits_dtype="bf16"),
+    Workload("wide_mha_b16_ragged", WIDE_MHA, batch=16, k=3, seed=2007, text_len_range=(2, 70),
+             logits_dtype="bf16"),
 ]}
 
 

@@ -27,6 +27,22 @@ def test_draft_kv_verify_parity_small(name, tc):
         case.close()
 
 
+@pytest.mark.parametrize("name", ["wide_gqa_b16_ragged", "wide_mha_b16_ragged"])
+def test_more_head_groups_than_attention_warps(name):
+    """16 sequences x 48 KV heads = 768 (sequence, head group) pairs against the 740 attention warps of the
+    tensor-core chain kernel: a warp takes several whole keys (head groups of 7), or a range of units that
+    spans several keys (single heads)."""
+    case = Case(hi.workload(name))
+    try:
+        case.drafter.set_tc_kernel(True)
+        res = check_draft_parity(case)
+        case.drafter.status()
+        check_kv_parity(case, res["ref"])
+        check_verify_parity(case, res["ids_o"])
+    finally:
+        case.close()
+
+
 def test_more_sequences_than_the_chain_kernels_take():
     """20 sequences: beyond the 16 of the tensor-core chain kernel, so the per-phase kernels run in two passes."""
     wl = hi.scaled(hi.workload("mini_gqa_b16_ragged"), batch=20, k=3, seed=2103)
