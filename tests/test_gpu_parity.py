@@ -43,6 +43,25 @@ def test_more_head_groups_than_attention_warps(name):
         case.close()
 
 
+@pytest.mark.parametrize("name", ["mini_gqa_b16_ragged", "mini_mha_b5_ragged", "wide_mha_b16_ragged"])
+def test_tensor_core_chain_kernel_repeats_bit_for_bit(name):
+    """Tiles shared between CTAs and keys shared between warps are summed in a fixed order whoever arrives
+    last, and the argmax is an integer maximum: two runs of the same draft give the same bits."""
+    case = Case(hi.workload(name))
+    try:
+        case.drafter.set_tc_kernel(True)
+        case.gpu_prefill()
+        ids_a, logits_a = case.gpu_draft()
+        for _ in range(3):
+            case.gpu_restore()
+            ids_b, logits_b = case.gpu_draft()
+            np.testing.assert_array_equal(ids_a, ids_b)
+            np.testing.assert_array_equal(logits_a.view(np.uint32), logits_b.view(np.uint32))
+        case.drafter.status()
+    finally:
+        case.close()
+
+
 def test_more_sequences_than_the_chain_kernels_take():
     """20 sequences: beyond the 16 of the tensor-core chain kernel, so the per-phase kernels run in two passes."""
     wl = hi.scaled(hi.workload("mini_gqa_b16_ragged"), batch=20, k=3, seed=2103)
