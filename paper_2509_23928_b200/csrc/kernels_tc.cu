@@ -16,7 +16,8 @@
 //   warps 4-7            epilogue: tcgen05.ld (one weight row per thread, 16 batch values), then the fused
 //                        output stage of the phase (residuals, RMSNorm statistics and gains, RoPE-free
 //                        QKV bias, SiLU*up, LM-head argmax keys) and the bf16 operand of the next phase.
-//   warps 3-7            between the QKV and O phases: split-KV attention over the text-only cache.  Its K/V
+//   warps 4-7            between the QKV and O phases: split-KV attention over the text-only cache (one warp per
+//                        scheduler: a fifth warp sharing a scheduler with another slowed both).  Its K/V
 //                        blocks travel through the same ring: the rows a sequence had when the launch began
 //                        do not change, so warp 0 copies them (between the QKV and the O tiles) ahead of the
 //                        grid barrier, and the attention warps compute from shared memory.
@@ -48,7 +49,8 @@
 #define TC_TN 16
 #define TC_A_BYTES (TC_TM * TC_BK * 2)
 #define TC_B_BYTES (TC_TN * TC_BK * 2)
-#define TC_ATT_WARPS 5               // warps 3..7 run the attention
+#define TC_ATT_FIRST 4               // first warp that runs the attention
+#define TC_ATT_WARPS (8 - TC_ATT_FIRST)
 #define TC_BAR_ATT 2
 #define TC_EPI_THREADS 128
 #define TC_BAR_EPI 3
@@ -1055,9 +1057,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
         if (lane == 0) tc_producer_x(P, ctl, smemB, cta, G, ai.total);
         __syncwarp();
     } else {
-        // warps 4..7: epilogue of every GEMM phase; warp 3: the embedding gather; warps 3..7: the attention
-        // between the QKV and O phases
-        const int atid = tid - 96;
+        // warps 4..7: epilogue of every GEMM phase and the attention between the QKV and O phases; warp 3: the
+        // embedding gather
+        const int atid = tid - 32 * TC_ATT_FIRST;        // < 0: not an attention warp
         const bool is_epi = warp >= 4;
         const int w4 = warp - 4;
         unsigned seg_cnt = 0;
@@ -1075,7 +1077,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
             if (p < PH_O) items_before += cnt;
         }
         TcAttRing ring;
-        ring.ctl = ctl; ring.error_flag = a.error_flag; ring.smemA = smemA; ring.w = warp - 3;
+        ring.ctl = ctl; ring.error_flag = a.error_flag; ring.smemA = smemA; ring.w = warp - TC_ATT_FIRST;
 #pragma unroll
         for (int w = 0; w < TC_ATT_WARPS; ++w) ring.n[w] = ai.n[w];
         for (int s = 0; s < a.k; ++s) {
@@ -1086,6 +1088,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
                 tc_gather(P, ctl, s, cta, G, lane);
             }
             // ---- attention: needs every CTA's QKV rows
+            if (atid < 0) continue;
             if (atid == 0)
                 wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(s * TC_BARS_PER_STEP + TC_SEQ_ATTN), ctl, a.error_flag, 7);
             named_sync(TC_BAR_ATT, TC_ATT_WARPS * 32);
@@ -1093,8 +1096,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
                 aw.step = s;
                 aw.rope_tab = a.rope_tab + (long long)(s & 1) * 16 * (DH / 2);
                 ring.base = items_before + (unsigned)s * items_step;
-                if constexpr (AttSel<GQ>::mma) attn_mma_phase<DH, GQ>(aw, ai.job[warp - 3], lane, ring);
-                else attn_warp_phase<DH, GQ>(aw, ai.pl, (warp - 3) * G + cta, lane, ring);
+                if constexpr (AttSel<GQ>::mma) attn_mma_phase<DH, GQ>(aw, ai.job[warp - TC_ATT_FIRST], lane, ring);
+                else attn_warp_phase<DH, GQ>(aw, ai.pl, (warp - TC_ATT_FIRST) * G + cta, lane, ring);
             }
             named_sync(TC_BAR_ATT, TC_ATT_WARPS * 32);
             if (atid == 0) {
