@@ -62,6 +62,36 @@ def test_tensor_core_chain_kernel_repeats_bit_for_bit(name):
         case.close()
 
 
+EDGE = [  # (base workload, batch, k, shortest and longest text length)
+    ("wide_mha_b16_ragged", 16, 2, 1, 1),            # no prefix at all: every key is its tail unit only
+    ("mini_gqa_b16_ragged", 3, 16, 1, 1),            # ... and the longest chain (16 appended rows)
+    ("mini_mha_b5_ragged", 5, 1, 32, 32),            # prefix of 31 rows: one block, not full
+    ("mini_gqa_b16_ragged", 16, 5, 33, 33),          # prefix of exactly one block
+    ("mini_mha_b5_ragged", 9, 8, 31, 34),            # lengths around the block boundary
+    ("wide_gqa_b16_ragged", 16, 16, 127, 129),       # several whole keys per warp, long chain
+    ("mini_gqa_b16_ragged", 2, 8, 1, 200),           # two sequences: keys cut into many parts
+    ("mini_mha_b5_ragged", 3, 5, 300, 300),          # long uniform prefixes, few keys
+    ("wide_mha_b16_ragged", 9, 16, 1, 90),
+]
+
+
+@pytest.mark.parametrize("base,batch,k,lo,hi_len", EDGE)
+def test_tensor_core_chain_kernel_edge_lengths(base, batch, k, lo, hi_len):
+    """Cache lengths at and around the 32-row block boundaries of the attention, an empty prefix, the
+    longest chain: the tensor-core chain kernel against the oracle."""
+    wl = hi.scaled(hi.workload(base), batch=batch, k=k, seed=9100 + batch + k + lo, text_len=None,
+                   text_len_range=(lo, hi_len))
+    case = Case(wl, max_k=16)
+    try:
+        case.drafter.set_tc_kernel(True)
+        res = check_draft_parity(case)
+        case.drafter.status()
+        check_kv_parity(case, res["ref"])
+        check_verify_parity(case, res["ids_o"])
+    finally:
+        case.close()
+
+
 def test_more_sequences_than_the_chain_kernels_take():
     """20 sequences: beyond the 16 of the tensor-core chain kernel, so the per-phase kernels run in two passes."""
     wl = hi.scaled(hi.workload("mini_gqa_b16_ragged"), batch=20, k=3, seed=2103)
