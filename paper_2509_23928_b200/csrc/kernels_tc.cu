@@ -891,6 +891,14 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
         }
     }
     if (lo < hi && big) named_sync(TC_BAR_EPI, TC_EPI_THREADS);
+    if (need_scale && lo < hi) {
+        // The RMSNorm scale of this phase's operand: wait here for the phase that produced it (rather than for
+        // the first accumulator, which for a short range is also the last: the sums would be fetched in the tail)
+        if (etid == 0) wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(need_seq(s, p) + 1), ctl, a.error_flag, 18);
+        named_sync(TC_BAR_EPI, TC_EPI_THREADS);
+        epi_compute_scales(a, ctl, p == PH_QKV ? a.ssq1 : a.ssq2, etid);
+        need_scale = false;
+    }
     const int tile_first = (int)(lo / sh.nkb);
     while (idx < hi) {
         const int tile = (int)(idx / sh.nkb), kb0 = (int)(idx % sh.nkb);
