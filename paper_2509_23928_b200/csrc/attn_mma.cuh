@@ -380,18 +380,16 @@ __device__ void attn_mma_phase(const AttnWArgs& a, const AttmJob& jb, int lane, 
                 __stcg((float2*)(a.part_acc + pi * DH + 8 * jn + 2 * t), make_float2(o[jn][0] + o[jn][2], o[jn][1] + o[jn][3]));
             if (t == 0) __stcg((float2*)(a.part_ml + pi * 2), make_float2(m_run, l_run));
         }
-        __threadfence();
         __syncwarp();
         int last = 0;
         if (lane == 0) {
             int* ctr = a.counters + b_cur * HG + hg_cur;
-            const int old = atomicAdd(ctr, nblk);
+            const int old = atom_add_acq_rel(ctr, nblk);
             last = (old + nblk == nb_cur);
             if (last) *ctr = 0;
         }
         last = __shfl_sync(0xffffffffu, last, 0);
         if (!last) continue;
-        __threadfence();
         // merge the key's parts in order: first the largest of their maxima, then one pass over the parts whose
         // loads do not depend on each other
         if (head_ok) {

@@ -124,6 +124,13 @@ __device__ __forceinline__ void attw_cursor_next(AttwCursor& c, const int* pos0,
     }
 }
 
+// arrival on a counter: orders this thread's writes, and those of threads it synchronised with before, ahead of
+// the addition (release) and the writes of earlier arrivers ahead of what follows (acquire), in one operation
+__device__ __forceinline__ int atom_add_acq_rel(int* p, int v) {
+    int old;
+    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
 __device__ __forceinline__ void attw_sts16(uint32_t addr, uint4 v) {
     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
@@ -425,18 +432,16 @@ __device__ void attn_warp_phase(const AttnWArgs& a, const AttwPlan& pl, int gw, 
                 __stcg(a.part_ml + pi * 2 + 1, l_run[g]);
             }
         }
-        __threadfence();
         __syncwarp();
         int last = 0;
         if (lane == 0) {
             int* ctr = a.counters + b_cur * HG + hg_cur;
-            const int old = atomicAdd(ctr, nblk);
+            const int old = atom_add_acq_rel(ctr, nblk);
             last = (old + nblk == nb_cur);
             if (last) *ctr = 0;
         }
         last = __shfl_sync(0xffffffffu, last, 0);
         if (!last) continue;
-        __threadfence();
         // merge the key's partials in block order (a partial starts where a warp's range meets the key), one
         // pass with running rescaling, all heads of the group per partial
         float M[GQ], L[GQ], A[GQ][EPL];

@@ -920,7 +920,6 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
         if (shared && big && idx != lo && hi - lo >= sh.nkb) {
             if (etid == 0) {
                 const int seen = ld_acquire_int(a.tile_ctr + tile);
-                __threadfence();
                 ctl->early_flag = seen == nc - 1;
             }
             named_sync(TC_BAR_EPI, TC_EPI_THREADS);
@@ -958,13 +957,11 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
                     const long long t0 = (long long)tile * sh.nkb;
                     for (long long i = t0; i < t0 + sh.nkb; ++nc) i = range_lo(sh.W, owner_of(sh.W, G, i) + 1, G);
                 }
-                __threadfence();                       // the CTA's partial (ordered before by the barrier) is visible first
-                const int old = atomicAdd(a.tile_ctr + tile, 1);
+                // release: the CTA's partial (ordered before by the barrier) is visible first; acquire: so are
+                // the partials of those that arrived before
+                const int old = atom_add_acq_rel(a.tile_ctr + tile, 1);
                 const int last = old == nc - 1;
-                if (last) {
-                    a.tile_ctr[tile] = 0;
-                    __threadfence();
-                }
+                if (last) a.tile_ctr[tile] = 0;
                 ctl->last_flag = last;
             }
             named_sync(TC_BAR_EPI, TC_EPI_THREADS);
