@@ -13,6 +13,13 @@ struct AttnSmem {
     int s_last;
 };
 
+// arrival on a counter: orders this thread's writes, and those of threads it synchronised with before, ahead of
+// the addition (release) and the writes of earlier arrivers ahead of what follows (acquire), in one operation
+__device__ __forceinline__ int atom_add_acq_rel(int* p, int v) {
+    int old;
+    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
 // cos/sin of pos * inv_freq: the product and its reduction to [-pi, pi] are done in double (a few
 // instructions), the functions themselves in fp32 on the reduced argument.
 __device__ __forceinline__ void rope_cs(int pos, double inv_freq, float& c, float& s) {
@@ -245,17 +252,15 @@ __device__ __forceinline__ void attn_unit(const AttnArgs& a, int split, int hg, 
     }
     if (single) return;
     // arrival counter: the last unit of this (sequence, head group) merges the splits; nobody waits
-    __threadfence();
     attn_sync<BAR, NT>();
     if (tid == 0) {
         int* ctr = a.counters + (long long)b * a.Hq + h0;
-        const int old = atomicAdd(ctr, 1);
+        const int old = atom_add_acq_rel(ctr, 1);
         sm.s_last = (old == nsplits - 1);
         if (sm.s_last) *ctr = 0;
     }
     attn_sync<BAR, NT>();
     if (!sm.s_last) return;
-    __threadfence();
     for (int i = tid; i < GQ * DH; i += NT) {
         const int gq = i / DH, dd = i % DH;
         const int h = h0 + gq;

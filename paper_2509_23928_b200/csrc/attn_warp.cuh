@@ -124,13 +124,6 @@ __device__ __forceinline__ void attw_cursor_next(AttwCursor& c, const int* pos0,
     }
 }
 
-// arrival on a counter: orders this thread's writes, and those of threads it synchronised with before, ahead of
-// the addition (release) and the writes of earlier arrivers ahead of what follows (acquire), in one operation
-__device__ __forceinline__ int atom_add_acq_rel(int* p, int v) {
-    int old;
-    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
-    return old;
-}
 __device__ __forceinline__ void attw_sts16(uint32_t addr, uint4 v) {
     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
