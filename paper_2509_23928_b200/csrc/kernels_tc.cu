@@ -596,7 +596,6 @@ __device__ void tc_gather(const TcParams& P, TcCtl* ctl, int s, int cta, int G, 
     }
     __syncwarp();
     if (lane == 0) {
-        fence_proxy_async_all();
         red_release_add_u64(a.bar_counter, 1ull);
     }
     __syncwarp();
@@ -1003,7 +1002,6 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
         const int need = p == PH_FC ? s * TC_BARS_PER_STEP + TC_SEQ_GATHER : need_seq(s, p);
         if ((lo == hi || p == PH_FC) && need >= 0)
             wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(need + 1), ctl, a.error_flag, 8);
-        fence_proxy_async_all();
         red_release_add_u64(a.bar_counter, 1ull);
     }
     // Without work in the phase nothing but the wait above tells this CTA that the earlier phases are complete:
@@ -1106,7 +1104,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
             }
             named_sync(TC_BAR_ATT, TC_ATT_WARPS * 32);
             if (atid == 0) {
-                fence_proxy_async_all();
                 red_release_add_u64(a.bar_counter, 1ull);
             }
             if (is_epi) {
