@@ -136,6 +136,8 @@ __device__ __forceinline__ void prefetch_tensormap(const void* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+// the same for global memory only: between an acquire and tiled copies of what other CTAs wrote
+__device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -536,7 +538,7 @@ __device__ void tc_producer_x(const TcParams& P, TcCtl* ctl, uint32_t smemB, int
             if (need >= 0) {
                 if (!wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(need + 1), ctl, a.error_flag, 9)) break;
                 // other CTAs wrote the operand through the generic proxy; TMA reads through the async proxy
-                fence_proxy_async_all();
+                fence_proxy_async_global();
             }
         }
         const bool emb = c.p == PH_FC && c.kb >= dkb;
@@ -544,7 +546,7 @@ __device__ void tc_producer_x(const TcParams& P, TcCtl* ctl, uint32_t smemB, int
             if (!wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(c.step * TC_BARS_PER_STEP + TC_SEQ_GATHER + 1), ctl,
                            a.error_flag, 11))
                 break;
-            fence_proxy_async_all();
+            fence_proxy_async_global();
             gathered_step = c.step;
         }
         if (round > 0 && !wait_mbar(saddr(&ctl->empty[slot]), (round - 1) & 1u, ctl, a.error_flag, 10)) break;
