@@ -30,8 +30,8 @@ import hivis_inputs as hi  # noqa: E402
 # DRAM bytes (read + written) of ONE launch of the chain kernel, from the ncu captures summarised under
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum).  Keyed by workload; a workload without a capture,
 # or a kernel that changed since, reports null.
-NCU_TRAFFIC = {"c2_llava_b1": 3672459000 + 4513280, "c5a_llava_b16_text_only": 3732340480 + 5461760,
-               "c4_qwen_b8": 11266300416 + 18955008}
+NCU_TRAFFIC = {"c2_llava_b1": 3672459000 + 4513280, "c5a_llava_b16_text_only": 3732322048 + 6112768,
+               "c4_qwen_b8": 11265867008 + 19566336}
 
 METRIC = "draft_steps_per_s"
 UNIT = "draft steps/s"
