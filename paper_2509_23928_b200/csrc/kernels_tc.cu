@@ -26,8 +26,9 @@
 // into equal contiguous ranges, one per CTA (so every SM streams the same number of bytes whatever the
 // matrix shape).  A tile that straddles CTAs is finished by whichever contributor arrives last: everyone
 // writes its partial accumulator to global scratch and bumps the tile's arrival counter; the last one adds
-// the partials in contributor order (fixed, so results do not depend on timing) and runs the output stage.
-// Nobody waits for anybody inside a phase.
+// the partials in a fixed order (so results do not depend on timing) and runs the output stage.  Where a
+// range is at least a tile long, the tile at its end is finished from an early look at the counter (the other
+// contributors did their part at the start of the phase).  Nobody waits for anybody inside a phase.
 //
 // Batch operand: activations are rounded to bf16 for the MMA; for B <= 8 the rounding remainder is fed
 // through the unused columns (rows [B, 2B) of every operand buffer) and added in the output stage, which
