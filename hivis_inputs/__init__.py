@@ -111,6 +111,14 @@ MINI_MHA = DrafterDims(d=512, n_q_heads=4, n_kv_heads=4, head_dim=128, ffn=1376,
 MINI_GQA = DrafterDims(d=448, n_q_heads=7, n_kv_heads=1, head_dim=64, ffn=1184, vocab=5031,
                        rms_eps=1e-6, dtype="bf16")
 
+# Head groups of 2, 4 and 8 query heads per KV head (the Qwen shape has 7).
+GQA2 = DrafterDims(d=512, n_q_heads=8, n_kv_heads=4, head_dim=64, ffn=1024, vocab=3001,
+                   rms_eps=1e-6, dtype="bf16")
+GQA4 = DrafterDims(d=512, n_q_heads=8, n_kv_heads=2, head_dim=128, ffn=1024, vocab=3001,
+                   rms_eps=1e-6, dtype="bf16")
+GQA8 = DrafterDims(d=512, n_q_heads=8, n_kv_heads=1, head_dim=64, ffn=1024, vocab=3001,
+                   rms_eps=1e-6, dtype="bf16")
+
 # Many heads at a small width: more (sequence, head group) pairs than a B200 has attention warps (740).
 WIDE_GQA = DrafterDims(d=128, n_q_heads=336, n_kv_heads=48, head_dim=64, ffn=256, vocab=1000,
                        rms_eps=1e-6, dtype="bf16")
@@ -140,6 +148,10 @@ WORKLOADS: Dict[str, Workload] = {w.name: w for w in [
              logits_dtype="bf16"),
     Workload("wide_mha_b16_ragged", WIDE_MHA, batch=16, k=3, seed=2007, text_len_range=(2, 70),
              logits_dtype="bf16"),
+    Workload("gqa2_b5_ragged", GQA2, batch=5, k=4, seed=2008, text_len_range=(1, 140), logits_dtype="bf16"),
+    Workload("gqa4_b16_ragged", GQA4, batch=16, k=3, seed=2009, text_len_range=(2, 100), logits_dtype="bf16"),
+    Workload("gqa8_b16_ragged", GQA8, batch=16, k=3, seed=2010, text_len_range=(2, 100), logits_dtype="f32"),
+    Workload("gqa4_b5_ragged", GQA4, batch=5, k=4, seed=2011, text_len_range=(1, 140), logits_dtype="bf16"),
 ]}
 
 

@@ -113,6 +113,9 @@ int hivis_destroy(hivis_ctx* ctx);
  * start_pos_host: NULL appends after the rows the slot holds now; otherwise start_pos_host[b]
  * (0 <= start <= current length) first truncates the slot to that many rows, which lets the
  * caller overwrite rows that came from drafting by rows built from true target features.
+ * A slot whose pending pair has not been drafted yet cannot be appended to (STATE): the row
+ * of that pair was never cached, so the new rows would land one position too early.  Pass the
+ * whole continuation in one call, or pass start_pos and repeat the pair.
  * resid0: [d] in ctx dtype = the initial residual r^0 (projected by resid_proj when the
  * context has one); NULL = no residual.
  * Errors: ARG, STATE, CAPACITY (rows + T_b - 1 + max... > max_len), CUDA.                    */
@@ -168,8 +171,11 @@ int hivis_read_kv(hivis_ctx* ctx, int slot, int row0, int n, float* out_k, float
 
 /* Debug: copy an intermediate of the LAST draft step of the last hivis_draft call, fp32,
  * [B, width] in call order: U fused input (d), ATTN attention output (n_q_heads*head_dim),
- * Y post-attention residual (d), ACT SwiGLU product (ffn), G layer output (d).               */
-enum { HIVIS_TAP_U = 0, HIVIS_TAP_ATTN = 1, HIVIS_TAP_Y = 2, HIVIS_TAP_ACT = 3, HIVIS_TAP_G = 4 };
+ * Y post-attention residual (d), ACT SwiGLU product (ffn), G layer output (d), Q the query
+ * projection with its bias and BEFORE the rotary embedding (n_q_heads*head_dim).  The K and V
+ * rows of that step are the slot's newest cache rows: read them with hivis_read_kv (K after
+ * the rotary embedding, as stored).                                                          */
+enum { HIVIS_TAP_U = 0, HIVIS_TAP_ATTN = 1, HIVIS_TAP_Y = 2, HIVIS_TAP_ACT = 3, HIVIS_TAP_G = 4, HIVIS_TAP_Q = 5 };
 int hivis_debug_tap(hivis_ctx* ctx, int which, float* out, void* stream);
 
 /* Options.
@@ -190,9 +196,13 @@ int hivis_debug_tap(hivis_ctx* ctx, int which, float* out, void* stream);
 enum { HIVIS_OPT_CHAIN_KERNEL = 0, HIVIS_OPT_TC_KERNEL = 1, HIVIS_OPT_WAIT_LIMIT_US = 2, HIVIS_OPT_DEBUG_MISS_BARRIER = 3 };
 int hivis_set_option(hivis_ctx* ctx, int option, int value);
 
-/* Synchronises `stream` and reports whether any kernel since the last call gave up on a bounded
- * device-side wait (HIVIS_ERR_TIMEOUT; the outputs of that call are invalid, the context stays
- * usable).  Otherwise HIVIS_OK.                                                                 */
+/* Synchronises `stream` and reports what the kernels since the last call recorded:
+ * HIVIS_ERR_TIMEOUT - a kernel gave up on a bounded device-side wait (the outputs of that call
+ *   are invalid, the context stays usable);
+ * HIVIS_ERR_ARG - a token id outside [0, vocab) reached the embedding lookup (ids passed to
+ *   hivis_prefill, forced_ids of hivis_draft; they live in device memory, so the host cannot
+ *   check them): the kernels read it as token 0 and went on, nothing faulted.
+ * Otherwise HIVIS_OK.  The record is cleared by the call.                                       */
 int hivis_status(hivis_ctx* ctx, void* stream);
 
 /* Per-kernel timing of hivis_draft.  Between hivis_profile_begin and hivis_profile_end every

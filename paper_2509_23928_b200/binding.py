@@ -10,7 +10,7 @@ LIB_PATH = os.path.join(HERE, "libhivis.so")
 
 HIVIS_F32, HIVIS_BF16 = 0, 1
 HIVIS_MAX_BATCH, HIVIS_MAX_K = 64, 16
-TAPS = {"u": 0, "attn": 1, "y": 2, "act": 3, "g": 4}
+TAPS = {"u": 0, "attn": 1, "y": 2, "act": 3, "g": 4, "q": 5}
 ERRORS = {0: "OK", -1: "ARG", -2: "SHAPE", -3: "DTYPE", -4: "STATE", -5: "CAPACITY", -6: "CUDA",
           -7: "TIMEOUT", -8: "NOMEM"}
 
@@ -279,7 +279,7 @@ class Drafter:
     def tap(self, name, B):
         t = self.torch
         width = {"u": self.dims.d, "attn": self.dims.n_q_heads * self.dims.head_dim, "y": self.dims.d,
-                 "act": self.dims.ffn, "g": self.dims.d}[name]
+                 "act": self.dims.ffn, "g": self.dims.d, "q": self.dims.n_q_heads * self.dims.head_dim}[name]
         out = t.empty((B, width), dtype=t.float32, device=self.dev)
         hivis_debug_tap(self.ctx, TAPS[name], out)
         return out

@@ -40,7 +40,8 @@ struct hivis_ctx {
     bool opt_chain;               // option HIVIS_OPT_CHAIN_KERNEL
     u64* bar_counter;
     u64 bar_count_host;           // value of *bar_counter once everything enqueued has run
-    int* error_flag;
+    int* error_flag;              // [0]: a device-side wait ran out; [1] (= id_flag): a token id was out of range
+    int* id_flag;
     // tensor-core chain kernel (bf16, up to 16 sequences)
     bool tc_ok;                   // cooperative launch available, shapes supported, tensor maps built
     long long wait_cycles;        // option HIVIS_OPT_WAIT_LIMIT_US, in cycles
@@ -292,7 +293,7 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
          dalloc(c, &c->part_acc, R * cfg->n_q_heads * (long long)c->nsplit_cap * cfg->head_dim) &&
          dalloc(c, &c->part_ml, R * cfg->n_q_heads * (long long)c->nsplit_cap * 2) &&
          dalloc(c, &c->counters, R * cfg->n_q_heads) && dalloc(c, &c->bar_counter, 1) &&
-         dalloc(c, &c->error_flag, 1) && dalloc(c, &c->slot_of, c->map_cap) &&
+         dalloc(c, &c->error_flag, 2) && dalloc(c, &c->slot_of, c->map_cap) &&
          dalloc(c, &c->row_of, c->map_cap) && dalloc(c, &c->xe_h, R * d) &&
          dalloc(c, &c->rope_tab, 2 * 16 * (cfg->head_dim / 2));
     if (!ok) {
@@ -302,6 +303,7 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
     }
     c->embed = embed; c->lm_head = lm; c->fc = fc; c->norm1 = n1; c->wqkv = wqkv; c->bqkv = bqkv;
     c->wo = wo; c->norm2 = n2; c->wgu = wgu; c->wdown = wdown; c->resid_proj = rp; c->Kc = Kc; c->Vc = Vc;
+    c->id_flag = c->error_flag + 1;
 
     int rc = HIVIS_OK;
     auto run = [&]() -> int {
@@ -334,7 +336,7 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
         CK(c, cudaMemsetAsync(c->pend_id, 0, MB * sizeof(int), st));
         CK(c, cudaMemsetAsync(c->counters, 0, R * cfg->n_q_heads * sizeof(int), st));
         CK(c, cudaMemsetAsync(c->bar_counter, 0, sizeof(u64), st));
-        CK(c, cudaMemsetAsync(c->error_flag, 0, sizeof(int), st));
+        CK(c, cudaMemsetAsync(c->error_flag, 0, 2 * sizeof(int), st));
         CK(c, cudaMemsetAsync(c->xe_h, 0, R * d * sizeof(bf16), st));
         CK(c, cudaMemsetAsync(c->feat_h, 0, R * d * sizeof(bf16), st));
         CK(c, cudaMemsetAsync(c->xq, 0, R * d * sizeof(bf16), st));
@@ -426,7 +428,7 @@ static void fill_chain_args(hivis_ctx* c, ChainArgs* a) {
     a->u = c->u; a->qkv = c->qkv; a->attn = c->attn; a->y = c->y; a->act = c->act; a->feat = c->feat;
     a->keys = c->keys; a->Kc = c->Kc; a->Vc = c->Vc; a->inv_freq = c->inv_freq;
     a->part_acc = c->part_acc; a->part_ml = c->part_ml; a->counters = c->counters;
-    a->bar_counter = c->bar_counter; a->error_flag = c->error_flag;
+    a->bar_counter = c->bar_counter; a->error_flag = c->error_flag; a->id_flag = c->id_flag;
 }
 
 static bool use_mma(const hivis_ctx* c, int B, bool prefill) {
@@ -440,7 +442,7 @@ static int run_fuse(hivis_ctx* c, bool mma, int b0, int nb, const float* feat, c
     LinArgs a;
     memset(&a, 0, sizeof(a));
     a.W = c->fc; a.N = d; a.K = 2 * d; a.B = nb; a.ldb = c->rows_cap; a.d = d;
-    a.feat = feat; a.feat_h = feat_h; a.embed = c->embed;
+    a.feat = feat; a.feat_h = feat_h; a.embed = c->embed; a.vocab = c->cfg.vocab; a.id_flag = c->id_flag;
     a.ids = ids; a.id_stride = id_stride; a.keys = keys; a.key_stride = c->key_stride;
     a.rho = rho;
     a.out = c->u + (long long)b0 * d;
@@ -497,6 +499,9 @@ int hivis_prefill(hivis_ctx* c, int B, const int* seq_slots_host, const int32_t*
         const int s = sl.slot[b];
         int base = c->kv_upper[s];
         start.slot[b] = -1;
+        if (!start_pos_host && c->pending[s])
+            return fail(c, HIVIS_ERR_STATE, "slot %d still holds a pending pair whose K/V row was never cached: draft it "
+                        "first, or pass start_pos to rebuild the rows from there", s);
         if (start_pos_host) {
             if (start_pos_host[b] < 0 || start_pos_host[b] > c->kv_upper[s])
                 return fail(c, HIVIS_ERR_ARG, "start_pos %d outside [0,%d]", start_pos_host[b], c->kv_upper[s]);
@@ -601,7 +606,7 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
         const int lo = B <= 8 ? 1 : 0;
         CKP(c, CLS_OTHER, st, launch_tc_setup(sl, k, d, lo, c->d_slots, c->d_pos0, c->kv_len, c->pend_feat, c->pend_id,
                                               c->feat, c->feat_h, c->cur_id, c->keys, c->key_stride, (const bf16*)c->embed,
-                                              V, c->xe_h, st));
+                                              V, c->xe_h, c->id_flag, st));
         ChainArgs ca;
         fill_chain_args(c, &ca);
         TcArgs a;
@@ -623,7 +628,7 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
         a.counters = c->counters;
         a.attn_nslot = c->nsplit_cap;
         a.bar_counter = c->bar_counter; a.bar_base = c->bar_count_host + (c->debug_skew ? (1ull << 40) : 0ull);
-        a.wait_cycles = c->wait_cycles; a.error_flag = c->error_flag;
+        a.wait_cycles = c->wait_cycles; a.error_flag = c->error_flag; a.id_flag = c->id_flag;
         c->debug_skew = false;
         CKP(c, CLS_CHAIN, st, launch_tc_chain(c->tc_maps, a, c->num_sms, st));
         c->bar_count_host += (u64)c->num_sms * (u64)(tc_barriers_per_step() * k);
@@ -844,13 +849,19 @@ int hivis_set_option(hivis_ctx* c, int option, int value) {
 int hivis_status(hivis_ctx* c, void* stream) {
     if (!c) return HIVIS_ERR_ARG;
     cudaStream_t st = (cudaStream_t)stream;
-    int flag = 0;
-    CK(c, cudaMemcpyAsync(&flag, c->error_flag, sizeof(int), cudaMemcpyDeviceToHost, st));
+    int flags[2] = {0, 0};
+    CK(c, cudaMemcpyAsync(flags, c->error_flag, 2 * sizeof(int), cudaMemcpyDeviceToHost, st));
     CK(c, cudaStreamSynchronize(st));
-    if (flag == 0) return HIVIS_OK;
+    const int flag = flags[0];
+    if (flag == 0 && flags[1] == 0) return HIVIS_OK;
+    if (flag == 0) {
+        CK(c, cudaMemsetAsync(c->id_flag, 0, sizeof(int), st));
+        CK(c, cudaStreamSynchronize(st));
+        return fail(c, HIVIS_ERR_ARG, "a token id outside [0, vocab) reached the embedding lookup and was read as token 0");
+    }
     // a kernel gave up on a wait: bring the barrier bookkeeping back to a known state
     CK(c, cudaMemsetAsync(c->bar_counter, 0, sizeof(u64), st));
-    CK(c, cudaMemsetAsync(c->error_flag, 0, sizeof(int), st));
+    CK(c, cudaMemsetAsync(c->error_flag, 0, 2 * sizeof(int), st));
     CK(c, cudaMemsetAsync(c->counters, 0, (size_t)c->rows_cap * c->cfg.n_q_heads * sizeof(int), st));
     if (c->tile_ctr) CK(c, cudaMemsetAsync(c->tile_ctr, 0, (size_t)c->tc_tiles * sizeof(int), st));
     CK(c, cudaStreamSynchronize(st));
@@ -894,6 +905,11 @@ int hivis_debug_tap(hivis_ctx* c, int which, float* out, void* stream) {
         case HIVIS_TAP_ATTN: src = c->attn; n = B * c->qw; break;
         case HIVIS_TAP_Y: src = c->y; n = B * d; break;
         case HIVIS_TAP_G: src = c->feat; n = B * d; break;
+        case HIVIS_TAP_Q:
+            // q sits at the start of every row of the stacked q | k | v buffer
+            CK(c, cudaMemcpy2DAsync(out, (size_t)c->qw * sizeof(float), c->qkv, (size_t)c->qkvw * sizeof(float),
+                                    (size_t)c->qw * sizeof(float), (size_t)B, cudaMemcpyDeviceToDevice, st));
+            return HIVIS_OK;
         case HIVIS_TAP_ACT:
             n = B * F;
             if (c->tap_mma) {

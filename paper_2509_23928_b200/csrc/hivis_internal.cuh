@@ -10,6 +10,8 @@
 typedef __nv_bfloat16 bf16;
 typedef unsigned long long u64;
 
+#define HIVIS_MAX_DEVICES 64   // per-device caches of function attributes are indexed by device ordinal
+
 // ---------------------------------------------------------------------------------------------
 // Skinny linear layer  out[b][n] = sum_k W[n][k] * x[b][k]  with a fused input stage (PRO_*)
 // and a fused output stage (EPI_*).  Two kernel families share these arguments:
@@ -36,6 +38,8 @@ struct LinArgs {
     const u64* keys;      // PRO_FUSE: packed argmax keys, row b at keys[b * key_stride]
     int key_stride;
     int d;
+    int vocab;            // PRO_FUSE: ids outside [0, vocab) are read as token 0 and raise *id_flag
+    int* id_flag;
     // ---- scale recovered from per-tile partial sums of squares (mma EPI_QKV / EPI_GATEUP):
     //      s[b] = rsqrt( sum_t ssq_in[t*ldb + b] / K + eps )
     const float* ssq_in;
@@ -121,6 +125,7 @@ struct ChainArgs {
     u64 bar_base;              // its value when this launch starts
     long long wait_cycles;     // limit of every device-side wait, in SM clock cycles
     int* error_flag;           // set non-zero by a kernel that gave up on a wait
+    int* id_flag;              // set non-zero when a token id outside [0, V) reached the embedding lookup
     int off_x, off_part, off_bar, off_misc;   // shared-memory layout, filled by the launcher
 };
 // shared memory the kernel needs for these dimensions on `grid` CTAs; 0 = does not fit
@@ -165,7 +170,7 @@ struct TcArgs {
     int key_stride;
     float *u, *qkv, *attn, *y, *feat;     // fp32 activations [B][width]
     bf16 *feat_h, *xq_h, *attn_h, *xm_h, *act_h;   // bf16 operands [TC_OP_ROWS][width]
-    bf16* xe_h;                // [TC_OP_ROWS][d] embedding rows of the step's tokens (rows >= B stay zero)
+    bf16* xe_h;                // [TC_OP_ROWS][d] embedding rows of the step's tokens (the set-up kernel zeroes rows >= B)
     const bf16* embed;         // [V][d]
     float *ssq1, *ssq2;        // [tiles*4][16] partial sums of squares of u / y
     float* logits_out;         // [B][k][V], nullable
@@ -181,6 +186,7 @@ struct TcArgs {
     u64 bar_base;
     long long wait_cycles;     // limit of every device-side wait, in SM clock cycles
     int* error_flag;
+    int* id_flag;              // set non-zero when a token id outside [0, V) reached the embedding lookup
 };
 // fills `maps` for the given buffers; returns cudaSuccess or an error (driver entry point missing, bad shape)
 cudaError_t tc_build_maps(TcMaps* maps, const ChainPhase* ph, int d, int qw, int F, const bf16* feat_h,
@@ -192,7 +198,7 @@ cudaError_t launch_tc_chain(const TcMaps& maps, const TcArgs& a, int grid, cudaS
 cudaError_t launch_tc_setup(const SlotList& sl, int k, int d, int lo, int* d_slots, int* d_pos0, int* kv_len,
                             const float* pend_feat, const int* pend_id, float* feat, bf16* feat_h,
                             int* cur_id, u64* keys, int key_stride, const bf16* embed, int vocab, bf16* xe_h,
-                            cudaStream_t st);
+                            int* id_flag, cudaStream_t st);
 int tc_barriers_per_step();
 
 // ---------------------------------------------------------------------------------------------
@@ -252,6 +258,13 @@ __device__ __forceinline__ u64 pack_key(float v, int idx) {
 }
 __device__ __forceinline__ int key_index(u64 key) {
     return (int)(0xFFFFFFFFu - (unsigned int)(key & 0xFFFFFFFFull));
+}
+// A token id on its way to the embedding table: an id outside [0, vocab) is read as token 0 and recorded in
+// *id_flag (reported by hivis_status), so that no lookup leaves the table whatever sits in device memory.
+__device__ __forceinline__ int checked_token(int id, int vocab, int* id_flag) {
+    if (id >= 0 && id < vocab) return id;
+    if (id_flag) *(volatile int*)id_flag = 1;
+    return 0;
 }
 __device__ __forceinline__ float bf16_lo(unsigned int w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(unsigned int w) { return __uint_as_float(w & 0xFFFF0000u); }

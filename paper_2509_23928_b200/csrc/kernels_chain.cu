@@ -298,6 +298,7 @@ __global__ void __launch_bounds__(CHAIN_THREADS, 1) draft_chain_kernel(const Cha
             if (s == 0) tok = a.pend_id[slot];
             else if (a.forced) tok = a.forced[s - 1];
             else tok = key_index(__ldcg(a.keys + (s - 1)));
+            tok = checked_token(tok, a.V, a.id_flag);
             const float* f = s == 0 ? a.pend_feat + (long long)slot * d : a.feat;
             const long long e0 = (long long)tok * d;
             for (int kk = tid; kk < K; kk += CHAIN_THREADS)
@@ -479,11 +480,15 @@ int chain_barriers_per_step() { return 7; }
 
 template <typename WT, int DH>
 static cudaError_t chain_launch_t(ChainArgs& a, int grid, size_t smem, cudaStream_t st) {
-    static size_t attr_smem = 0;
-    if (smem > attr_smem) {
+    // the shared-memory opt-in is a per-device attribute of the function: remember it per device ordinal
+    static size_t attr_smem[HIVIS_MAX_DEVICES] = {0};
+    int dev = 0;
+    cudaError_t e0 = cudaGetDevice(&dev);
+    if (e0 != cudaSuccess) return e0;
+    if (dev < 0 || dev >= HIVIS_MAX_DEVICES || smem > attr_smem[dev]) {
         cudaError_t e = cudaFuncSetAttribute(draft_chain_kernel<WT, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        attr_smem = smem;
+        if (dev >= 0 && dev < HIVIS_MAX_DEVICES) attr_smem[dev] = smem;
     }
     void* params[] = {(void*)&a};
     return cudaLaunchCooperativeKernel((const void*)draft_chain_kernel<WT, DH>, dim3(grid), dim3(CHAIN_THREADS), params, smem, st);

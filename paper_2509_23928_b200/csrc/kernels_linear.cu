@@ -68,8 +68,8 @@ __device__ __forceinline__ void epilogue_pair(const LinArgs& a, int b, int row, 
 }
 
 __device__ __forceinline__ int fuse_token(const LinArgs& a, int b) {
-    if (a.ids) return a.ids[(long long)b * a.id_stride];
-    return key_index(a.keys[(long long)b * a.key_stride]);
+    const int id = a.ids ? a.ids[(long long)b * a.id_stride] : key_index(a.keys[(long long)b * a.key_stride]);
+    return checked_token(id, a.vocab, a.id_flag);
 }
 
 // ==========================================================================================
@@ -225,13 +225,17 @@ __global__ void __launch_bounds__(256) gemv_alu_kernel(const LinArgs a, int ppw)
 
 template <typename WT, int PRO, int EPI>
 static cudaError_t launch_alu_t(const LinArgs& a, cudaStream_t st) {
-    static bool attr_set = false;
+    // the shared-memory opt-in is a per-device attribute of the function: remember it per device ordinal
+    static bool attr_set[HIVIS_MAX_DEVICES] = {false};
     const size_t smem = (size_t)a.K * sizeof(float);
-    if (!attr_set) {
+    int dev = 0;
+    cudaError_t e0 = cudaGetDevice(&dev);
+    if (e0 != cudaSuccess) return e0;
+    if (dev < 0 || dev >= HIVIS_MAX_DEVICES || !attr_set[dev]) {
         cudaError_t e = cudaFuncSetAttribute(gemv_alu_kernel<WT, PRO, EPI>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        if (dev >= 0 && dev < HIVIS_MAX_DEVICES) attr_set[dev] = true;
     }
     if (smem > 200 * 1024) return cudaErrorInvalidValue;
     const long long pairs = ((long long)a.N + 1) / 2;

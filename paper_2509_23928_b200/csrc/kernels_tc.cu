@@ -217,20 +217,20 @@ __device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, TcCtl* 
 // The count is a plain shared-memory word written after the arming by the same thread: operations of one
 // thread on the CTA's shared memory (the barrier's arrive included) take effect in program order, so a reader
 // that sees the count finds the barrier armed.  (A release/acquire pair here costs a fence per ring item.)
-__device__ __forceinline__ unsigned ld_acquire_cta_u32(const unsigned* p) {
+__device__ __forceinline__ unsigned ld_volatile_cta_u32(const unsigned* p) {
     unsigned v;
     asm volatile("ld.volatile.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(saddr(p)) : "memory");
     return v;
 }
-__device__ __forceinline__ void st_release_cta_u32(unsigned* p, unsigned v) {
+__device__ __forceinline__ void st_volatile_cta_u32(unsigned* p, unsigned v) {
     asm volatile("st.volatile.shared::cta.u32 [%0], %1;" ::"r"(saddr(p)), "r"(v) : "memory");
 }
 __device__ __forceinline__ bool wait_issued(TcCtl* ctl, unsigned idx, int* error_flag, int code) {
     if (poisoned(ctl)) return false;
-    if ((int)(ld_acquire_cta_u32(&ctl->issued) - idx) > 0) return true;
+    if ((int)(ld_volatile_cta_u32(&ctl->issued) - idx) > 0) return true;
     const long long t0 = clock64();
     unsigned it = 0;
-    while ((int)(ld_acquire_cta_u32(&ctl->issued) - idx) <= 0) {
+    while ((int)(ld_volatile_cta_u32(&ctl->issued) - idx) <= 0) {
         if ((++it & 63u) == 0u) {
             if (poisoned(ctl)) return false;
             if (ld_relaxed_int(error_flag) != 0) { *(volatile int*)&ctl->abort_flag = 1; return false; }
@@ -456,7 +456,7 @@ __device__ bool tc_issue_attention(const TcParams& P, TcCtl* ctl, uint32_t smemA
             if constexpr (AttSel<GQ>::mma) attm_cursor_next(cur[w], a.pos0, a.slots, HG);
             else attw_cursor_next(cur[w], a.pos0, HG);
             if (++slot == TC_STAGES) { slot = 0; ++round; }
-            st_release_cta_u32(&ctl->issued, round * TC_STAGES + slot);
+            st_volatile_cta_u32(&ctl->issued, round * TC_STAGES + slot);
         }
     }
     return true;
@@ -503,7 +503,7 @@ __device__ void tc_producer_w(const TcParams& P, TcCtl* ctl, uint32_t smemA, int
         cursor_next(c, a, cta, G);
         if (++slot == TC_STAGES) { slot = 0; ++round; }
         if (publish) {
-            st_release_cta_u32(&ctl->issued, round * TC_STAGES + slot);
+            st_volatile_cta_u32(&ctl->issued, round * TC_STAGES + slot);
             --publish;
         }
     }
@@ -591,7 +591,7 @@ __device__ void tc_gather(const TcParams& P, TcCtl* ctl, int s, int cta, int G, 
                 const int b = i / upr, off = i - b * upr;
                 int id = a.forced ? __ldcg(a.forced + (long long)b * a.k + (s - 1))
                                   : key_index(__ldcg(a.keys + (long long)b * a.key_stride + (s - 1)));
-                if (id < 0 || id >= a.V) id = 0;
+                id = checked_token(id, a.V, a.id_flag);
                 const uint4 w = ld_stream((const uint4*)(a.embed + (long long)id * a.d) + off);
                 __stcg((uint4*)(a.xe_h + (long long)b * a.d) + off, w);
             }
@@ -1129,8 +1129,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
 // ------------------------------------------------------------------------------------------ set-up kernel
 __global__ void tc_setup_kernel(SlotList sl, int k, int d, int lo, int* d_slots, int* d_pos0, int* kv_len,
                                 const float* pend_feat, const int* pend_id, float* feat, bf16* feat_h, int* cur_id,
-                                u64* keys, int key_stride, const bf16* embed, int vocab, bf16* xe_h) {
-    const int b = blockIdx.x, slot = sl.slot[b];
+                                u64* keys, int key_stride, const bf16* embed, int vocab, bf16* xe_h, int* id_flag) {
+    const int b = blockIdx.x;
+    if (b >= sl.n) {
+        // Rows of the embedding operand beyond the batch: the tiled copy always brings all 16 rows, and for B <= 8
+        // accumulator columns [B, 2B) are added to columns [0, B) as rounding remainders (an embedding row is exact
+        // in bf16, so its remainder is zero).  An earlier, larger batch may have left rows here.
+        for (int i = threadIdx.x; i < (d >> 3); i += blockDim.x)
+            ((uint4*)(xe_h + (long long)b * d))[i] = make_uint4(0u, 0u, 0u, 0u);
+        return;
+    }
+    const int slot = sl.slot[b];
     if (threadIdx.x == 0) {
         d_slots[b] = slot;
         const int rows = kv_len[slot];
@@ -1147,16 +1156,16 @@ __global__ void tc_setup_kernel(SlotList sl, int k, int d, int lo, int* d_slots,
         if (lo) feat_h[(long long)(b + sl.n) * d + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
     }
     // embedding row of the pending token: the fusion FC's embedding operand of step 0
-    int id = pend_id[slot];
-    if (id < 0 || id >= vocab) id = 0;
+    const int id = checked_token(pend_id[slot], vocab, id_flag);
     for (int i = threadIdx.x; i < (d >> 3); i += blockDim.x)
         ((uint4*)(xe_h + (long long)b * d))[i] = ((const uint4*)(embed + (long long)id * d))[i];
 }
 cudaError_t launch_tc_setup(const SlotList& sl, int k, int d, int lo, int* d_slots, int* d_pos0, int* kv_len,
                             const float* pend_feat, const int* pend_id, float* feat, bf16* feat_h, int* cur_id,
-                            u64* keys, int key_stride, const bf16* embed, int vocab, bf16* xe_h, cudaStream_t st) {
-    tc_setup_kernel<<<sl.n, 256, 0, st>>>(sl, k, d, lo, d_slots, d_pos0, kv_len, pend_feat, pend_id, feat, feat_h,
-                                          cur_id, keys, key_stride, embed, vocab, xe_h);
+                            u64* keys, int key_stride, const bf16* embed, int vocab, bf16* xe_h, int* id_flag,
+                            cudaStream_t st) {
+    tc_setup_kernel<<<TC_OP_ROWS, 256, 0, st>>>(sl, k, d, lo, d_slots, d_pos0, kv_len, pend_feat, pend_id, feat, feat_h,
+                                                cur_id, keys, key_stride, embed, vocab, xe_h, id_flag);
     return cudaGetLastError();
 }
 
@@ -1235,13 +1244,17 @@ cudaError_t tc_build_maps(TcMaps* maps, const ChainPhase* ph, int d, int qw, int
 
 template <int DH, int GQ>
 static cudaError_t tc_launch_t(const TcParams& P, int grid, cudaStream_t st) {
-    static bool attr_set = false;
+    // the shared-memory opt-in is a per-device attribute of the function: remember it per device ordinal
+    static bool attr_set[HIVIS_MAX_DEVICES] = {false};
     const size_t smem = 1024 + (size_t)TC_STAGES * (TC_A_BYTES + TC_B_BYTES) + ((sizeof(TcCtl) + 127) & ~(size_t)127);
     if (smem > 227 * 1024) return cudaErrorInvalidValue;
-    if (!attr_set) {
+    int dev = 0;
+    cudaError_t e0 = cudaGetDevice(&dev);
+    if (e0 != cudaSuccess) return e0;
+    if (dev < 0 || dev >= HIVIS_MAX_DEVICES || !attr_set[dev]) {
         cudaError_t e = cudaFuncSetAttribute(tc_chain_kernel<DH, GQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        if (dev >= 0 && dev < HIVIS_MAX_DEVICES) attr_set[dev] = true;
     }
     void* params[] = {(void*)&P};
     return cudaLaunchCooperativeKernel((const void*)tc_chain_kernel<DH, GQ>, dim3(grid), dim3(TC_THREADS), params, smem, st);

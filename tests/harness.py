@@ -6,22 +6,11 @@ import numpy as np
 
 import hivis_inputs as hi
 import oracle
+from hivis_inputs.device import dev_weights, to_dev  # noqa: F401  (re-exported for the tests)
 
 LOGIT_RTOL = 2e-2          # max |gpu - ref| / max |ref| per logits row (bf16 storage, fp32 accumulation)
 LOGIT_RTOL_F32 = 2e-4      # fp32 workloads
 ID_GAP = 1e-2              # ids may differ only where the oracle's top-2 logit gap is below this
-
-
-def to_dev(arr, dtype: str):
-    import torch
-    arr = np.ascontiguousarray(arr, dtype=np.float32)
-    if dtype == "bf16":
-        return torch.from_numpy(hi.to_bf16_bits(arr).view(np.int16).reshape(arr.shape)).view(torch.bfloat16).cuda()
-    return torch.from_numpy(arr).cuda()
-
-
-def dev_weights(W, dtype: str):
-    return {n: to_dev(v, dtype) for n, v in W.items() if v is not None}
 
 
 class Case:

@@ -92,6 +92,122 @@ def test_tensor_core_chain_kernel_edge_lengths(base, batch, k, lo, hi_len):
         case.close()
 
 
+GROUPS = ["gqa2_b5_ragged", "gqa4_b16_ragged", "gqa8_b16_ragged", "gqa4_b5_ragged"]
+
+
+@pytest.mark.parametrize("tc", [True, False])
+@pytest.mark.parametrize("name", GROUPS)
+def test_head_groups_of_2_4_8(name, tc):
+    """2, 4 and 8 query heads per KV head, head dimensions 64 and 128, ragged batches of 5 and 16: in the
+    tensor-core chain kernel these run the single-head attention body with several query heads mapped onto one
+    KV head (the tensor-core attention body takes groups that are multiples of 7)."""
+    case = Case(hi.workload(name))
+    try:
+        case.drafter.set_tc_kernel(tc)
+        res = check_draft_parity(case)
+        case.drafter.status()
+        check_kv_parity(case, res["ref"])
+        check_verify_parity(case, res["ids_o"])
+    finally:
+        case.close()
+
+
+def test_smaller_batch_after_a_larger_one_on_the_same_context():
+    """A draft of 16 sequences followed, on the same context, by a draft of 4 of them: nothing the larger call
+    left in the operand buffers (embedding rows, rounding-remainder rows) may leak into the smaller one."""
+    import torch
+    wl = hi.workload("mini_gqa_b16_ragged")
+    case = Case(wl)
+    try:
+        case.drafter.set_tc_kernel(True)
+        ref = case.oracle_run()
+        ids_o = np.stack([r["ids"] for r in ref])
+        logits_o = np.stack([r["logits"] for r in ref])
+        case.gpu_prefill()
+        case.gpu_draft()                                   # all 16 sequences
+        case.gpu_restore()
+        sub = [9, 2, 14, 5]
+        f = torch.from_numpy(np.ascontiguousarray(ids_o[sub], np.int32)).cuda()
+        ids_g, logits_g = case.drafter.draft(len(sub), wl.k, case.d_resid, slots=sub, forced_ids=f, want_logits=True)
+        torch.cuda.synchronize()
+        case.drafter.status()
+        err = row_rel_err(logits_g.cpu().numpy(), logits_o[sub])
+        assert err.max() <= 2e-2, f"logits rel err {err.max()}"
+        # and bit for bit what a fresh context computes for the same four sequences
+        case2 = Case(wl)
+        try:
+            case2.drafter.set_tc_kernel(True)
+            case2.gpu_prefill()
+            ids_h, logits_h = case2.drafter.draft(len(sub), wl.k, case2.d_resid, slots=sub, forced_ids=f, want_logits=True)
+            torch.cuda.synchronize()
+            assert torch.equal(logits_g, logits_h) and torch.equal(ids_g, ids_h)
+        finally:
+            case2.close()
+    finally:
+        case.close()
+
+
+@pytest.mark.parametrize("name,tc,chain", [("mini_mha_b1", False, True), ("mini_mha_b1", False, False),
+                                           ("mini_mha_b5_ragged", True, True), ("mini_mha_b5_ragged", False, True)])
+def test_out_of_range_token_id_is_reported_not_followed(name, tc, chain):
+    """Token ids live in device memory, so only the kernels can check them.  A forced id beyond the vocabulary is
+    read as token 0 (no lookup leaves the embedding table), hivis_status reports HIVIS_ERR_ARG once, and the
+    logits are those of a chain fed token 0 at that step."""
+    from paper_2509_23928_b200 import HivisError
+    wl = hi.workload(name)
+    case = Case(wl)
+    try:
+        case.drafter.set_tc_kernel(tc)
+        case.drafter.set_chain_kernel(chain)
+        ref0 = case.oracle_run()
+        forced = np.stack([r["ids"] for r in ref0]).copy()
+        bad = forced.copy()
+        bad[wl.batch - 1, 1] = wl.dims.vocab + 12345         # consumed by step 2
+        if wl.batch > 1:
+            bad[0, 0] = -7
+        clean = bad.copy()
+        clean[(bad < 0) | (bad >= wl.dims.vocab)] = 0
+        ref = case.oracle_run(forced=clean)
+        case.gpu_prefill()
+        ids_g, logits_g = case.gpu_draft(forced=bad)
+        with pytest.raises(HivisError) as e:
+            case.drafter.status()
+        assert e.value.code == -1
+        case.drafter.status()                              # the record was cleared
+        err = row_rel_err(logits_g, np.stack([r["logits"] for r in ref]))
+        assert err.max() <= 2e-2
+        case.gpu_restore()
+        case.gpu_draft(forced=clean)
+        case.drafter.status()                              # valid ids: nothing to report
+    finally:
+        case.close()
+
+
+@pytest.mark.parametrize("name,tc", [("mini_mha_b1", False), ("mini_mha_b5_ragged", True), ("mini_mha_b5_ragged", False)])
+def test_nan_hidden_state_gives_token_zero_on_both_sides(name, tc):
+    """A NaN in the pending hidden state makes every logit of the chain NaN.  NaN never wins an argmax and an
+    all-NaN row gives index 0, on both sides; nothing is looked up outside the embedding table."""
+    import torch
+    wl = hi.workload(name)
+    case = Case(wl)
+    try:
+        case.drafter.set_tc_kernel(tc)
+        b = wl.batch - 1
+        last = int(case.cu[b + 1]) - 1
+        case.hidden[last, 3] = np.nan
+        case.d_hidden = to_dev(case.hidden, wl.dims.dtype)
+        ref = case.oracle_run(k=3)
+        assert (ref[b]["ids"] == 0).all() and np.isnan(ref[b]["logits"]).all()
+        case.gpu_prefill()
+        ids_g, logits_g = case.gpu_draft(3)
+        case.drafter.status()
+        assert (ids_g[b] == 0).all() and np.isnan(logits_g[b]).all()
+        for o in range(wl.batch - 1):                      # the other sequences are untouched
+            assert np.isfinite(logits_g[o]).all()
+    finally:
+        case.close()
+
+
 def test_more_sequences_than_the_chain_kernels_take():
     """20 sequences: beyond the 16 of the tensor-core chain kernel, so the per-phase kernels run in two passes."""
     wl = hi.scaled(hi.workload("mini_gqa_b16_ragged"), batch=20, k=3, seed=2103)
@@ -183,6 +299,16 @@ def test_intermediate_taps_match_oracle(tc):
                 got = case.drafter.tap(name, wl.batch)[b].cpu().numpy()
                 e = np.abs(got - taps[name]).max() / np.abs(taps[name]).max()
                 assert e < 2e-2, f"tap {name} seq {b}: rel err {e}"
+            # q leaves the library before the rotary embedding; the oracle's tap is taken after it
+            D = wl.dims
+            q_g = case.drafter.tap("q", wl.batch)[b].cpu().numpy()
+            q_rot = case.oracle.rope(q_g, D.n_q_heads, D.head_dim, D.rope_base, T - 1)
+            e = np.abs(q_rot - taps["q"]).max() / np.abs(taps["q"]).max()
+            assert e < 2e-2, f"tap q seq {b}: rel err {e}"
+            k_g, v_g = case.drafter.read_kv(b, T - 1, 1)       # the step's K (rotated) and V rows
+            for got, want, nm in ((k_g, taps["k"], "k"), (v_g, taps["v"], "v")):
+                e = np.abs(got[0].cpu().numpy() - want).max() / np.abs(want).max()
+                assert e < 2e-2, f"{nm} row of seq {b}: rel err {e}"
     finally:
         case.close()
 
@@ -405,6 +531,11 @@ def test_host_side_errors_do_not_launch():
         with pytest.raises(HivisError) as e:                     # second draft without a pending pair
             dr.draft(1, 4, case.d_resid)
         assert e.value.code == -4
+        case.gpu_restore()
+        n1 = dr.launch_count()
+        with pytest.raises(HivisError) as e:                     # appending while a pair is still pending
+            dr.prefill(case.d_ids, case.d_hidden, [0, 4])
+        assert e.value.code == -4 and dr.launch_count() == n1
     finally:
         case.close()
 
@@ -489,6 +620,16 @@ def test_full_size_c3_llava_b16_ragged_sampled():
 
 def test_full_size_c4_qwen_b8_sampled():
     _sampled_full_size("c4_qwen_b8", 2)
+
+
+def test_full_size_c5a_llava_b16_text_only_sampled():
+    _sampled_full_size("c5a_llava_b16_text_only", 2)
+
+
+def test_full_size_c5b_llava_b16_naive_kv_sampled():
+    """704 cached positions per sequence: 22 full blocks and a tail per key, uniform batch (the key-aligned
+    split of the attention units over the warps)."""
+    _sampled_full_size("c5b_llava_b16_naive_kv", 2)
 
 
 @pytest.mark.parametrize("name,tc", [("mini_mha_b1", False), ("mini_mha_b1", True), ("mini_gqa_b16_ragged", True)])

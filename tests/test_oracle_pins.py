@@ -377,6 +377,55 @@ def test_cache_rows_written_are_exactly_text_positions():
     assert written.tolist() == [True] * (T + k - 1) + [False] * 3      # n_cached == T + k - 1
 
 
+# ------------------------------------------------------------------ refresh of drafted rows (Alg. 1 line 9; Eq. 2)
+@pytest.mark.parametrize("n_new", [1, 2, 4])
+def test_prefill_at_a_start_position_equals_a_prefill_of_the_whole_pair_list(n_new):
+    """After a round the accepted tokens come back with TARGET features: every prefix position carries a target
+    feature and r^0 (Eq. 2), so rows T.. of the cache are rebuilt from true-feature pairs at their own positions.
+    Prefill T pairs, draft k (which fills rows T-1..T+k-2 with self-fed rows), refresh from start_pos = T - 1 with
+    the old pending pair followed by n_new new pairs; the next draft must equal the brute-force recompute and the
+    numpy restatement on the whole updated pair list.  A refresh that rotated K by p instead of start_pos + p, or
+    stored its rows at p, fails here."""
+    dims = small_dims(d=24, n_q_heads=4, n_kv_heads=2, head_dim=6, ffn=20, vocab=31)
+    W = rand_weights(dims, seed=41, scale=0.4, bias=True)
+    o = oracle.Oracle(dims, W)
+    rng = np.random.default_rng(42 + n_new)
+    T, k = 5, 4
+    ids = rng.integers(0, dims.vocab, T).astype(np.int32)
+    hidden = rng.standard_normal((T, dims.d)).astype(np.float32)
+    resid = rng.standard_normal((3, dims.d)).astype(np.float32)
+    rho = o.fold_residuals(resid)
+    Kc, Vc = o.new_cache(T + n_new + 2 * k)
+    o.prefill(ids, hidden, rho[0], Kc, Vc)
+    o.draft(T - 1, int(ids[-1]), hidden[-1], k, rho, Kc, Vc)             # rows T-1 .. T+k-2 now hold drafted rows
+    drafted_rows = Kc[T - 1:T + k - 1].copy()
+    new_ids = rng.integers(0, dims.vocab, n_new).astype(np.int32)
+    new_hidden = rng.standard_normal((n_new, dims.d)).astype(np.float32)
+    # the refresh: the old pending pair (its row was written by draft step 0 from the same inputs) and the new pairs
+    ref_ids = np.concatenate([ids[-1:], new_ids])
+    ref_hidden = np.concatenate([hidden[-1:], new_hidden])
+    o.prefill(ref_ids, ref_hidden, rho[0], Kc, Vc, start_pos=T - 1)
+    all_ids, all_hidden = np.concatenate([ids, new_ids]), np.concatenate([hidden, new_hidden])
+    L = T + n_new
+    # rows 0..L-2 are exactly those of one prefill of the whole list; rows beyond were not touched
+    K2, V2 = o.new_cache(T + n_new + 2 * k)
+    o.prefill(all_ids, all_hidden, rho[0], K2, V2)
+    np.testing.assert_array_equal(Kc[:L - 1], K2[:L - 1])
+    np.testing.assert_array_equal(Vc[:L - 1], V2[:L - 1])
+    if n_new < k:
+        np.testing.assert_array_equal(Kc[L - 1:T + k - 1], drafted_rows[n_new:])
+    if n_new > 1:                                    # the refreshed rows differ from the self-fed rows they replaced
+        assert np.abs(Kc[T:L - 1] - drafted_rows[1:n_new]).max() > 1e-3
+    # the next draft from the refreshed cache
+    got = o.draft(L - 1, int(all_ids[-1]), all_hidden[-1], k, rho, Kc, Vc)
+    bf = o.draft_bruteforce(all_ids, all_hidden, k, rho)
+    ref_tok, ref_logits = numpy_drafter(dims, W, all_ids, all_hidden, k, resid.astype(np.float64))
+    np.testing.assert_array_equal(got["ids"], bf["ids"])
+    np.testing.assert_array_equal(got["ids"], ref_tok)
+    np.testing.assert_allclose(got["logits"], bf["logits"], rtol=1e-10, atol=1e-11)
+    np.testing.assert_allclose(got["logits"], ref_logits, rtol=1e-9, atol=1e-10)
+
+
 # ------------------------------------------------------------------ verification (Sec. 2.1)
 def test_verify_all_match_patterns_bruteforce():
     dims = small_dims()

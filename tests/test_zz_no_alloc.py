@@ -1,4 +1,4 @@
-"""hivis_verify_noalloc against hivis_verify.
+"""hivis_verify_noalloc against hivis_verify and against the CPU oracle's verification.
 
 hivis_verify_noalloc is the greedy verification for callers that are not allowed to allocate device
 memory (a plug-in inside a server whose pool owns the GPU, code running after allocation has been
@@ -39,10 +39,13 @@ def test_noalloc_verify_matches_context_verify_twice_in_a_row(name):
         # two different sets of target logits: planted accept lengths, then heavy exact ties
         logits_a, planted = hi.make_target_logits(wl, ids_np)
         rng = np.random.default_rng(11)
-        logits_b = rng.integers(-3, 4, size=(B, k + 1, V)).astype(np.float32)
+        logits_b = rng.integers(-3, 4, size=(B, k + 1, V)).astype(np.float32)     # exact in bf16 too
         want_a = _reference_verify(case, d_ids, logits_a, wl)
         want_b = _reference_verify(case, d_ids, logits_b, wl)
         assert (want_a[0] == planted).all()
+        # what the oracle's greedy verification gives for each sequence (Sec. 2.1), independent of the CUDA path
+        oracle_a = [case.oracle.verify(ids_np[b], logits_a[b], int(case.lens[b])) for b in range(B)]
+        oracle_b = [case.oracle.verify(ids_np[b], logits_b[b], int(case.lens[b])) for b in range(B)]
 
         ldt = HIVIS_BF16 if wl.logits_dtype == "bf16" else HIVIS_F32
         rows_before = torch.from_numpy((case.lens - 1).astype(np.int32)).cuda()
@@ -52,10 +55,13 @@ def test_noalloc_verify_matches_context_verify_twice_in_a_row(name):
         for (acc, nxt, kv), d_log in zip(outs, (d_a, d_b, d_a)):
             hivis_verify_noalloc(B, k, V, d_ids, d_log, ldt, rows_before, acc, nxt, kv)
         torch.cuda.synchronize()
-        for (acc, nxt, kv), want in zip(outs, (want_a, want_b, want_a)):
-            np.testing.assert_array_equal(acc.cpu().numpy(), want[0])
-            np.testing.assert_array_equal(nxt.cpu().numpy(), want[1])
-            np.testing.assert_array_equal(kv.cpu().numpy(), want[2])
+        for (acc, nxt, kv), want, orc in zip(outs, (want_a, want_b, want_a), (oracle_a, oracle_b, oracle_a)):
+            acc, nxt, kv = acc.cpu().numpy(), nxt.cpu().numpy(), kv.cpu().numpy()
+            np.testing.assert_array_equal(acc, want[0])
+            np.testing.assert_array_equal(nxt, want[1])
+            np.testing.assert_array_equal(kv, want[2])
+            for b in range(B):
+                assert (int(acc[b]), int(nxt[b]), int(kv[b])) == orc[b], f"seq {b} against the oracle"
         # without the row counts
         acc, nxt = outs[0][0].fill_(-7), outs[0][1].fill_(-7)
         hivis_verify_noalloc(B, k, V, d_ids, d_b, ldt, None, acc, nxt, None)
