@@ -7,13 +7,23 @@ argmax) followed by batched greedy verification with KV rollback.  `value` count
 (k per benchmark step).  Inputs are seeded and synthetic; weights are random-init in the shape of
 the named backbone.
 
+The metric is quoted at batch 1 and batch 16.  Without --workload the run times the batch-1
+workload (the headline `value`, `roofline`, `e2e`) and then, in the same process, the batch-16
+workload with the text-only cache (key `batch16`: its own value, roofline, e2e and clock sample) and
+its naive-cache twin with 576 extra leading positions (key `batch16_naive_kv`: the ablation pair).
+
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+--gpus N > 1 means N independent replicas, one process per GPU (no collective on the path).  Under
+torchrun the ranks come from the environment; started plainly, the script launches its own N ranks.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
+import socket
 import subprocess
 import sys
 import threading
@@ -27,14 +37,12 @@ if ROOT not in sys.path:
 
 import hivis_inputs as hi  # noqa: E402
 
-# DRAM bytes (read + written) of ONE launch of the chain kernel, from the ncu captures summarised under
-# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum).  Keyed by workload; a workload without a capture,
-# or a kernel that changed since, reports null.
-NCU_TRAFFIC = {"c2_llava_b1": 3672459000 + 4513280, "c5a_llava_b16_text_only": 3732322048 + 6112768,
-               "c4_qwen_b8": 11265867008 + 19566336}
-
 METRIC = "draft_steps_per_s"
 UNIT = "draft steps/s"
+HEADLINE = "c2_llava_b1"
+BATCH16 = "c5a_llava_b16_text_only"
+BATCH16_NAIVE = "c5b_llava_b16_naive_kv"
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_traffic.json")
 
 
 def measured_peaks():
@@ -45,6 +53,29 @@ def measured_peaks():
         except Exception:
             pass
     return 6650.0, "fallback"
+
+
+def kernel_source_hash() -> str:
+    """Hash of the CUDA sources: ties a stored profiler figure to the kernels it was taken from."""
+    csrc = os.path.join(ROOT, "paper_2509_23928_b200", "csrc")
+    h = hashlib.sha256()
+    for name in sorted(os.listdir(csrc)):
+        if name.endswith((".cu", ".cuh")):
+            h.update(name.encode())
+            h.update(open(os.path.join(csrc, name), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def captured_traffic(workload: str):
+    """DRAM bytes (read + written) of ONE launch of the chain kernel on `workload`, from the ncu capture recorded
+    in profiles/ncu_traffic.json; None when there is no capture or the kernels have changed since it was taken."""
+    try:
+        rec = json.load(open(TRAFFIC_FILE))["captures"][workload]
+    except Exception:
+        return None
+    if rec.get("source_hash") != kernel_source_hash():
+        return None
+    return int(rec["dram_bytes_read"]) + int(rec["dram_bytes_write"])
 
 
 def max_over_ranks(value: float, dist, device: str) -> float:
@@ -66,6 +97,30 @@ def job_throughput(world: int, steps: int, k: int, slowest_ms: float) -> float:
 def replica_workload(wl, rank: int, world: int):
     """Replica `rank` of `world`: same shapes, its own seed (no data is shared, no collective on the path)."""
     return wl if world == 1 else hi.scaled(wl, seed=wl.seed + 100 * rank)
+
+
+def free_port() -> int:
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def spawn_replicas(n: int, argv) -> int:
+    """Start n ranks of this script (one per GPU) with the rendezvous variables torchrun would set; rank 0 prints
+    the job's line.  Returns the first non-zero exit code, else 0."""
+    port = free_port()
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__), *argv], env=env))
+    rc = 0
+    for p in procs:
+        p.wait()
+        rc = rc or p.returncode
+    return rc
 
 
 class ClockSampler:
@@ -145,64 +200,45 @@ def run_oracle_sample(wl, steps: int, warmup: int):
             "ms_per_bench_step": t / nseq * wl.batch * 1e3}
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=500)
-    ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2_llava_b1")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true")
-    args = ap.parse_args()
-    wl = hi.workload(args.workload)
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    config = {"workload": wl.name, "batch": wl.batch, "k": wl.k, "draft_steps_per_bench_step": wl.k,
-              "text_len": wl.text_len if wl.text_len else list(wl.text_len_range),
-              "leading_positions": wl.leading_positions, "d": wl.dims.d, "ffn": wl.dims.ffn,
-              "vocab": wl.dims.vocab, "heads": [wl.dims.n_q_heads, wl.dims.n_kv_heads, wl.dims.head_dim],
-              "logits_dtype": wl.logits_dtype, "parallelism": f"replicas x{args.gpus} (no collective)",
-              "l2": "weights streamed per step (>= 734 MB) exceed the 126 MB L2; no flush needed"}
+def workload_config(wl, world: int):
+    return {"workload": wl.name, "batch": wl.batch, "k": wl.k, "draft_steps_per_bench_step": wl.k,
+            "text_len": wl.text_len if wl.text_len else list(wl.text_len_range),
+            "leading_positions": wl.leading_positions, "d": wl.dims.d, "ffn": wl.dims.ffn,
+            "vocab": wl.dims.vocab, "heads": [wl.dims.n_q_heads, wl.dims.n_kv_heads, wl.dims.head_dim],
+            "logits_dtype": wl.logits_dtype, "parallelism": f"replicas x{world} (no collective)",
+            "l2": "weights streamed per step (>= 734 MB) exceed the 126 MB L2; no flush needed"}
 
-    if args.impl == "reference":
-        if rank != 0:
-            return
-        steps = max(1, min(args.steps, 3))
-        warm = max(1, min(args.warmup, 1))
-        cb = run_oracle_sample(wl, steps, warm)
-        line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": UNIT, "n_gpus": args.gpus,
-                "steps": steps, "warmup": warm, "ms_per_step": cb["ms_per_bench_step"], "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
-                "cpu_baseline": {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")},
-                "e2e": {"value": cb["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-                "gpu_launches": 0}
-        print(json.dumps(line))
-        return
 
+class WeightCache:
+    """Device weights per (dims, seed): the batch-16 workload and its naive-cache twin share one set."""
+
+    def __init__(self):
+        self.key, self.dW = None, None
+
+    def get(self, wl):
+        from hivis_inputs.device import dev_weights
+        key = (wl.dims, wl.seed)
+        if key != self.key:
+            self.dW = None
+            W = hi.make_weights(wl.dims, wl.seed)
+            self.dW = dev_weights(W, wl.dims.dtype)
+            self.key = key
+        return self.dW
+
+
+def time_workload(wl, steps: int, warmup: int, rank: int, local_rank: int, world: int, dist, weights: WeightCache,
+                  want_e2e: bool, short: bool = False):
+    """Prefill (untimed), then `steps` timed benchmark steps of `wl` on this rank's GPU.  Returns the pieces of the
+    JSON line that belong to one workload.  short=True: device timing of the chain only (no e2e, no clock sample)."""
     import torch
-    from paper_2509_23928_b200 import Drafter, hivis_profile_begin, hivis_profile_end
-    from tests.harness import to_dev, dev_weights  # device placement helpers only
-
-    assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback)"
-    torch.cuda.set_device(local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    wl = replica_workload(wl, rank, world)                 # independent replicas, same shapes
-
-    # ---------------- set-up (untimed): weights, prompt, prefill
-    W = hi.make_weights(wl.dims, wl.seed)
+    from hivis_inputs.device import to_dev
+    from paper_2509_23928_b200 import (Drafter, hivis_profile_begin, hivis_profile_end, hivis_verify, hivis_draft,
+                                       HIVIS_BF16, HIVIS_F32)
     ids, hidden, cu = hi.make_prompt(wl)
     resid = hi.make_residuals(wl)
     lens = np.diff(cu)
-    B, k, V = wl.batch, wl.k, wl.dims.vocab
-    dW = dev_weights(W, wl.dims.dtype)
-    del W
-    dr = Drafter(wl.dims, dW, max_batch=B, max_len=int(lens.max()) + k + 8, max_k=max(k, 8))
-    del dW
+    B, k = wl.batch, wl.k
+    dr = Drafter(wl.dims, weights.get(wl), max_batch=B, max_len=int(lens.max()) + k + 8, max_k=max(k, 8))
     torch.cuda.empty_cache()
     d_ids = torch.from_numpy(ids).cuda()
     d_hidden = to_dev(hidden, wl.dims.dtype)
@@ -217,7 +253,6 @@ def main():
     acc = torch.empty(B, dtype=torch.int32, device="cuda")
     nxt = torch.empty(B, dtype=torch.int32, device="cuda")
     kvl = torch.empty(B, dtype=torch.int32, device="cuda")
-    from paper_2509_23928_b200 import hivis_verify, hivis_draft, HIVIS_BF16, HIVIS_F32
     ldt = HIVIS_BF16 if wl.logits_dtype == "bf16" else HIVIS_F32
     stream = torch.cuda.current_stream()
 
@@ -236,15 +271,15 @@ def main():
 
     # ---------------- timed region: K steps, CUDA events on the launching stream
     sampler = ClockSampler(local_rank)
-    if rank == 0:
+    if rank == 0 and not short:
         sampler.start()
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(max(warmup, 3)):
         restore(); one_step()
     barrier()
     n0 = dr.launch_count()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    draft_ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    for i in range(args.steps):
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    draft_ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    for i in range(steps):
         restore()
         ev[i][0].record(stream)
         hivis_draft(dr.ctx, B, None, k, d_resid, d_resid.shape[0], out_ids, None, None, stream)
@@ -252,18 +287,19 @@ def main():
         hivis_verify(dr.ctx, B, None, k, out_ids, d_logits, ldt, acc, nxt, kvl, stream)
         ev[i][1].record(stream)
     barrier()
-    launches = dr.launch_count() - n0 - args.steps * B          # restore kernels sit outside the events
+    launches = dr.launch_count() - n0 - steps * B               # restore kernels sit outside the events
     step_ms = np.array([a.elapsed_time(b) for a, b in ev])
-    draft_ms = np.array([ev[i][0].elapsed_time(draft_ev[i]) for i in range(args.steps)])
+    draft_ms = np.array([ev[i][0].elapsed_time(draft_ev[i]) for i in range(steps)])
     total_ms = float(step_ms.sum())
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop() if (rank == 0 and not short) else None
     total_ms = max_over_ranks(total_ms, dist, "cuda")
     ok_planted = bool((acc.cpu().numpy() == planted).all())
+    dr.status()                                                  # no wait ran out, no id was out of range
 
     # ---------------- per-kernel device time (separate pass: events around every launch)
     restore()
     hivis_profile_begin(dr.ctx)
-    reps = min(args.steps, 20)
+    reps = min(steps, 20)
     for _ in range(reps):
         hivis_draft(dr.ctx, B, None, k, d_resid, d_resid.shape[0], out_ids, None, None, stream)
         restore()
@@ -283,7 +319,7 @@ def main():
             kern[name] = {"us": round(us, 2), "launches_per_draft_step": n // (reps * k),
                           "GBps": round(class_bytes[name] / (us * 1e-6) / 1e9, 1)}
     chain_ms, chain_n = prof.get("draft_chain", (0.0, 0))
-    if chain_n:                      # one sequence: the whole k-step chain is a single persistent kernel
+    if chain_n:                      # the whole k-step chain is a single persistent kernel
         us = chain_ms / chain_n * 1e3
         nbytes = k * step_bytes
         kern["draft_chain"] = {"us": round(us, 2), "launches_per_bench_step": 1,
@@ -296,7 +332,7 @@ def main():
         dom_bytes = class_bytes[dom]
     roofline = {"bound": "hbm", "kernel": dom, "achieved": kern[dom]["GBps"], "peak": peak, "unit": "GB/s",
                 "frac": round(kern[dom]["GBps"] / peak, 4), "peak_kind": peak_kind,
-                "traffic": NCU_TRAFFIC.get(wl.name) if (dom == "draft_chain" and world == 1) else None,
+                "traffic": captured_traffic(wl.name) if (dom == "draft_chain" and world == 1) else None,
                 "algorithmic_bytes_per_launch": dom_bytes, "per_kernel": kern}
 
     draft_us_per_step = float(np.median(draft_ms)) / k * 1e3
@@ -311,7 +347,7 @@ def main():
 
     # ---------------- end to end through the C ABI with HOST buffers
     e2e = None
-    if not args.no_e2e:
+    if want_e2e and not short:
         h_resid = d_resid.cpu().pin_memory()
         h_logits = d_logits.cpu().pin_memory()
         h_ids = torch.empty((B, k), dtype=torch.int32).pin_memory()
@@ -320,7 +356,7 @@ def main():
         d_res = torch.empty((3, Bp), dtype=torch.int32, device="cuda")
         d_resid2 = torch.empty_like(d_resid)
         d_logits2 = torch.empty_like(d_logits)
-        n_e2e = max(3, min(args.steps, 20))
+        n_e2e = max(3, min(steps, 20))
         barrier()
         t0 = time.perf_counter()
         for _ in range(n_e2e):
@@ -338,22 +374,118 @@ def main():
                "h2d_bytes_per_step": int(h_resid.numel() * h_resid.element_size() + h_logits.numel() * h_logits.element_size()),
                "d2h_bytes_per_step": int(h_ids.numel() * 4 + 3 * B * 4), "steps": n_e2e,
                "ms_per_step": t_e2e / n_e2e * 1e3}
+    dr.close()
+    return {"value": job_throughput(world, steps, k, total_ms), "ms_per_step": total_ms / steps, "clocks": clocks,
+            "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "draft_chain": chain,
+            "verify_matches_planted": ok_planted}
+
+
+def stub_replica(rank: int) -> dict:
+    """Stands in for the device work when HIVIS_BENCH_STUB=1 (CPU test of the launch path only): fixed fake
+    times, rank 1 slower.  The line it leads to is marked as a stub and carries no measurement."""
+    return {"total_ms": 10.0 + 5.0 * rank}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=None, help="time this workload only (default: batch 1, then batch 16)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.gpus < 1:
+        ap.error("--gpus must be at least 1")
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1 and args.impl == "ours":
+        sys.exit(spawn_replicas(args.gpus, sys.argv[1:]))          # one process per GPU; rank 0 prints the line
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "ours" and world != args.gpus:
+        sys.exit(f"bench.py: --gpus {args.gpus} but {world} rank(s) were started: refusing to report replicas that did not run")
+    wl = hi.workload(args.workload or HEADLINE)
+    config = workload_config(wl, world)
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        steps = max(1, min(args.steps, 3))
+        warm = max(1, min(args.warmup, 1))
+        cb = run_oracle_sample(wl, steps, warm)
+        line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": UNIT, "n_gpus": args.gpus,
+                "steps": steps, "warmup": warm, "ms_per_step": cb["ms_per_bench_step"], "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
+                "cpu_baseline": {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")},
+                "e2e": {"value": cb["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line))
+        return
+
+    stub = os.environ.get("HIVIS_BENCH_STUB") == "1"
+    if stub:
+        import torch.distributed as dist
+        if world > 1:
+            dist.init_process_group("gloo", rank=rank, world_size=world)
+        slowest = max_over_ranks(stub_replica(rank)["total_ms"], dist if world > 1 else None, "cpu")
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": None, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                              "data": "stub (no device work: launch-path test)", "config": config,
+                              "stub_slowest_ms": slowest}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    import torch
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    wl = replica_workload(wl, rank, world)                 # independent replicas, same shapes
+    weights = WeightCache()
+    res = time_workload(wl, args.steps, args.warmup, rank, local_rank, world, dist, weights, not args.no_e2e)
+
+    extra = {}
+    if args.workload is None:
+        # the batch-16 half of the metric, and the visual-token-hiding pair (text-only cache vs naive cache)
+        w16 = replica_workload(hi.workload(BATCH16), rank, world)
+        r16 = time_workload(w16, args.steps, args.warmup, rank, local_rank, world, dist, weights, not args.no_e2e)
+        r16["config"] = workload_config(w16, world)
+        wnv = replica_workload(hi.workload(BATCH16_NAIVE), rank, world)
+        rnv = time_workload(wnv, min(args.steps, 100), args.warmup, rank, local_rank, world, dist, weights, False,
+                            short=True)
+        a, b = r16["draft_chain"], rnv["draft_chain"]
+        extra["batch16"] = r16
+        extra["batch16_naive_kv"] = {
+            "workload": wnv.name, "leading_positions": wnv.leading_positions,
+            "us_per_draft_step": b["us_per_draft_step_median"], "GBps": b["GBps"], "frac_of_peak": b["frac_of_peak"],
+            "algorithmic_bytes_per_draft_step": b["algorithmic_bytes_per_draft_step"],
+            "roofline_frac": rnv["roofline"]["frac"], "kernel_us_per_launch": rnv["roofline"]["per_kernel"].get("draft_chain", {}).get("us"),
+            "text_only_us_per_draft_step": a["us_per_draft_step_median"],
+            "naive_over_text_only": round(b["us_per_draft_step_median"] / a["us_per_draft_step_median"], 4),
+            "verify_matches_planted": rnv["verify_matches_planted"]}
+    weights = None
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        dr.close()
+        torch.cuda.empty_cache()
         cb = run_oracle_sample(wl, 3, 1)
         cpu_baseline = {k_: cb[k_] for k_ in ("value", "unit", "cores", "kind", "sample")}
         cpu_baseline["us_per_step"] = round(cb["us_per_step"], 1)
 
     if rank == 0:
-        line = {"metric": METRIC, "value": job_throughput(world, args.steps, k, total_ms), "unit": UNIT,
+        D = wl.dims
+        line = {"metric": METRIC, "value": res["value"], "unit": UNIT,
                 "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-                "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+                "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16 storage, f32 accumulate" if D.dtype == "bf16" else "f32",
-                "data": "synthetic", "config": config, "clocks": clocks, "e2e": e2e,
-                "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu_baseline,
-                "draft_chain": chain, "verify_matches_planted": ok_planted}
+                "data": "synthetic", "config": config, "clocks": res["clocks"], "e2e": res["e2e"],
+                "gpu_launches": res["gpu_launches"], "roofline": res["roofline"], "cpu_baseline": cpu_baseline,
+                "draft_chain": res["draft_chain"], "verify_matches_planted": res["verify_matches_planted"]}
+        line.update(extra)
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

@@ -30,6 +30,8 @@ struct hivis_ctx {
     bf16 *feat_h, *xq, *attn_h, *xm, *act_h;
     u64* keys;
     int key_stride;
+    u64* vkeys;                   // verification: argmax keys [max_batch][max_k + 1] and arrival counters
+    int* varrive;                 // [max_batch]; both zero between calls
     float *part_acc, *part_ml;
     int* counters;
     int chunk, nsplit_cap;
@@ -290,6 +292,7 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
          dalloc(c, &c->act_h, R * F) && dalloc(c, &c->rho_raw, (long long)HIVIS_MAX_K * d) &&
          dalloc(c, &c->rho, (long long)HIVIS_MAX_K * d) && dalloc(c, &c->ssq1, tiles1 * R) &&
          dalloc(c, &c->ssq2, tiles1 * R) && dalloc(c, &c->keys, R * c->key_stride) &&
+         dalloc(c, &c->vkeys, MB * (cfg->max_k + 1)) && dalloc(c, &c->varrive, MB) &&
          dalloc(c, &c->part_acc, R * cfg->n_q_heads * (long long)c->nsplit_cap * cfg->head_dim) &&
          dalloc(c, &c->part_ml, R * cfg->n_q_heads * (long long)c->nsplit_cap * 2) &&
          dalloc(c, &c->counters, R * cfg->n_q_heads) && dalloc(c, &c->bar_counter, 1) &&
@@ -337,6 +340,8 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
         CK(c, cudaMemsetAsync(c->counters, 0, R * cfg->n_q_heads * sizeof(int), st));
         CK(c, cudaMemsetAsync(c->bar_counter, 0, sizeof(u64), st));
         CK(c, cudaMemsetAsync(c->error_flag, 0, 2 * sizeof(int), st));
+        CK(c, cudaMemsetAsync(c->vkeys, 0, MB * (cfg->max_k + 1) * sizeof(u64), st));
+        CK(c, cudaMemsetAsync(c->varrive, 0, MB * sizeof(int), st));
         CK(c, cudaMemsetAsync(c->xe_h, 0, R * d * sizeof(bf16), st));
         CK(c, cudaMemsetAsync(c->feat_h, 0, R * d * sizeof(bf16), st));
         CK(c, cudaMemsetAsync(c->xq, 0, R * d * sizeof(bf16), st));
@@ -764,7 +769,7 @@ int hivis_verify(hivis_ctx* c, int B, const int* seq_slots_host, int k, const in
             return fail(c, HIVIS_ERR_STATE, "slot %d: verify(k=%d) must follow a draft of the same k", sl.slot[b], k);
     cudaStream_t st = (cudaStream_t)stream;
     int nl = 0;
-    CK(c, launch_verify(logits_dtype, sl, k, c->cfg.vocab, draft_ids, target_logits, c->keys, c->kv_len,
+    CK(c, launch_verify(logits_dtype, sl, k, c->cfg.vocab, draft_ids, target_logits, c->vkeys, c->varrive, c->kv_len,
                         out_accept, out_next, out_kv_len, st, &nl));
     c->launches += nl;
     for (int b = 0; b < B; ++b) {

@@ -230,9 +230,10 @@ cudaError_t launch_kv_append(int dtype, const float* kv /*[P][2*kvw]*/, int P, c
                              const int* row_of, const double* inv_freq, int Hkv, int dh, int max_len,
                              void* Kc, void* Vc, cudaStream_t st);
 
-// verification: row argmax over [B][k+1][V], then accept length / next token / rollback
+// verification in one launch: row argmax over [B][k+1][V], accept length / next token / rollback.
+// keys [B][k+1] and arrivals [B] must be zero on entry and are left zero.
 cudaError_t launch_verify(int logits_dtype, const SlotList& sl, int k, int V, const int32_t* draft_ids,
-                          const void* logits, u64* keys, int* kv_len, int32_t* out_accept,
+                          const void* logits, u64* keys, int* arrivals, int* kv_len, int32_t* out_accept,
                           int32_t* out_next, int32_t* out_kv_len, cudaStream_t st, int* n_launches);
 
 cudaError_t launch_set_int(int* p, int v, cudaStream_t st);

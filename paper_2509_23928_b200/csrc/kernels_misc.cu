@@ -149,14 +149,23 @@ cudaError_t launch_kv_append(int dtype, const float* kv, int P, const int* slot_
 }
 
 // ------------------------------------------------------------------------------------------
-// greedy verification: row argmax, then accept length / next token / rollback
+// greedy verification in one launch: row argmax over [B][k+1][V], accept length, next token, rollback
 // ------------------------------------------------------------------------------------------
 #define VERIFY_CHUNK 8192   // logits per CTA
 
+// One CTA per (chunk of a row, row, sequence).  Every CTA folds its chunk into the row's packed argmax key
+// (integer max: lowest index among equal values, independent of arrival order) and counts itself on the
+// sequence's arrival counter; the CTA that completes the count reads the sequence's k + 1 keys, finds the
+// longest accepted prefix, writes the outputs, rolls the slot back, and leaves keys and counter zero for the
+// next call.  Nobody waits.
 template <typename LT>
-__global__ void __launch_bounds__(256) verify_argmax_kernel(const void* logits, int V, u64* keys) {
+__global__ void __launch_bounds__(256) verify_kernel(SlotList sl, int k, const void* logits, int V,
+                                                     const int32_t* draft_ids, u64* keys, int* arrivals,
+                                                     int* kv_len, int32_t* out_accept, int32_t* out_next,
+                                                     int32_t* out_kv_len) {
     __shared__ u64 kred[8];
-    const long long rowi = (long long)blockIdx.z * gridDim.y + blockIdx.y;   // b*(k+1) + j
+    const int b = blockIdx.z;
+    const long long rowi = (long long)b * (k + 1) + blockIdx.y;
     const LT* row = (const LT*)logits + rowi * V;
     const int c0 = blockIdx.x * VERIFY_CHUNK;
     const int c1 = min(V, c0 + VERIFY_CHUNK);
@@ -200,43 +209,40 @@ __global__ void __launch_bounds__(256) verify_argmax_kernel(const void* logits, 
     }
     if ((threadIdx.x & 31) == 0) kred[threadIdx.x >> 5] = best;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        u64 m = kred[0];
+    if (threadIdx.x != 0) return;
+    u64 m = kred[0];
 #pragma unroll
-        for (int w = 1; w < 8; ++w) m = kred[w] > m ? kred[w] : m;
-        if (m) atomicMax(keys + rowi, m);
-    }
-}
-
-__global__ void verify_finish_kernel(SlotList sl, int k, const int32_t* draft_ids, const u64* keys,
-                                     int* kv_len, int32_t* out_accept, int32_t* out_next,
-                                     int32_t* out_kv_len) {
-    const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= sl.n) return;
-    const u64* kr = keys + (long long)b * (k + 1);
+    for (int w = 1; w < 8; ++w) m = kred[w] > m ? kred[w] : m;
+    atomicMax(keys + rowi, m);
+    // release: the key update above is visible before the count; acquire: so are those of earlier arrivers
+    const int total = (int)gridDim.x * (k + 1);
+    if (atom_add_acq_rel(arrivals + b, 1) != total - 1) return;
+    u64* kr = keys + (long long)b * (k + 1);
     int n = 0;
-    while (n < k && key_index(kr[n]) == draft_ids[(long long)b * k + n]) ++n;
+    while (n < k && key_index(__ldcg(kr + n)) == draft_ids[(long long)b * k + n]) ++n;
+    const int next = key_index(__ldcg(kr + n));
     const int slot = sl.slot[b];
     const int pairs = kv_len[slot] - k + 1;          // true-feature pairs of the sequence
     const int rows = pairs + (n < k - 1 ? n : k - 1);
     kv_len[slot] = rows;
     out_accept[b] = n;
-    out_next[b] = key_index(kr[n]);
+    out_next[b] = next;
     if (out_kv_len) out_kv_len[b] = rows;
+    for (int j = 0; j <= k; ++j) kr[j] = 0ull;
+    arrivals[b] = 0;
 }
 
 cudaError_t launch_verify(int logits_dtype, const SlotList& sl, int k, int V, const int32_t* draft_ids,
-                          const void* logits, u64* keys, int* kv_len, int32_t* out_accept,
+                          const void* logits, u64* keys, int* arrivals, int* kv_len, int32_t* out_accept,
                           int32_t* out_next, int32_t* out_kv_len, cudaStream_t st, int* n_launches) {
-    cudaError_t e = cudaMemsetAsync(keys, 0, sizeof(u64) * sl.n * (k + 1), st);
-    if (e != cudaSuccess) return e;
     dim3 grid((unsigned)((V + VERIFY_CHUNK - 1) / VERIFY_CHUNK), (unsigned)(k + 1), (unsigned)sl.n);
-    if (logits_dtype == HIVIS_BF16) verify_argmax_kernel<bf16><<<grid, 256, 0, st>>>(logits, V, keys);
-    else verify_argmax_kernel<float><<<grid, 256, 0, st>>>(logits, V, keys);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    verify_finish_kernel<<<1, 64, 0, st>>>(sl, k, draft_ids, keys, kv_len, out_accept, out_next, out_kv_len);
-    *n_launches = 2;
+    if (logits_dtype == HIVIS_BF16)
+        verify_kernel<bf16><<<grid, 256, 0, st>>>(sl, k, logits, V, draft_ids, keys, arrivals, kv_len, out_accept,
+                                                   out_next, out_kv_len);
+    else
+        verify_kernel<float><<<grid, 256, 0, st>>>(sl, k, logits, V, draft_ids, keys, arrivals, kv_len, out_accept,
+                                                    out_next, out_kv_len);
+    *n_launches = 1;
     return cudaGetLastError();
 }
 

@@ -47,3 +47,39 @@ def test_reference_arm_prints_one_line_from_rank_zero_only():
     p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2"],
                        capture_output=True, text=True, env=env, timeout=120)
     assert p.returncode == 0 and p.stdout.strip() == ""
+
+
+def test_plain_launch_with_gpus_2_starts_two_ranks_itself():
+    """`python bench.py --gpus 2` outside torchrun: the script starts its own two ranks (here on gloo with the device
+    work stubbed), both go through the rank reduction, rank 0 prints one line with n_gpus = 2."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    env["HIVIS_BENCH_STUB"] = "1"
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "4"],
+                       capture_output=True, text=True, env=env, timeout=300)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [l for l in p.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["config"]["parallelism"].startswith("replicas x2")
+    assert line["stub_slowest_ms"] == 15.0 and line["value"] is None and "stub" in line["data"]
+
+
+def test_fewer_ranks_than_gpus_is_refused():
+    """--gpus 8 with a single started rank must not print a line that claims eight replicas."""
+    env = dict(os.environ, RANK="0", LOCAL_RANK="0", WORLD_SIZE="1", HIVIS_BENCH_STUB="1")
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "8"],
+                       capture_output=True, text=True, env=env, timeout=120)
+    assert p.returncode != 0 and p.stdout.strip() == "" and "refusing" in p.stderr
+
+
+def test_traffic_figure_is_dropped_when_the_kernels_changed(tmp_path, monkeypatch):
+    import bench
+    f = tmp_path / "t.json"
+    good = {"captures": {"w": {"dram_bytes_read": 10, "dram_bytes_write": 5, "source_hash": bench.kernel_source_hash()}}}
+    f.write_text(json.dumps(good))
+    monkeypatch.setattr(bench, "TRAFFIC_FILE", str(f))
+    assert bench.captured_traffic("w") == 15
+    assert bench.captured_traffic("other") is None
+    good["captures"]["w"]["source_hash"] = "0" * 16
+    f.write_text(json.dumps(good))
+    assert bench.captured_traffic("w") is None
