@@ -232,7 +232,7 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
     c->qw = cfg->n_q_heads * cfg->head_dim;
     c->kvw = cfg->n_kv_heads * cfg->head_dim;
     c->qkvw = c->qw + 2 * c->kvw;
-    c->rows_cap = cfg->max_batch > 16 ? cfg->max_batch : 16;
+    c->rows_cap = cfg->max_batch > TC_OP_ROWS ? cfg->max_batch : TC_OP_ROWS;
     c->launches = 0;
     c->err[0] = 0;
     c->tap_B = 0;
@@ -608,7 +608,7 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
     }
     if (c->tc_ok && c->opt_tc != 0 && B <= 16) {
         // bf16, up to 16 sequences: all k steps in one cooperative tensor-core kernel
-        const int lo = B <= 8 ? 1 : 0;
+        const int lo = tc_lo_offset(B);
         CKP(c, CLS_OTHER, st, launch_tc_setup(sl, k, d, lo, c->d_slots, c->d_pos0, c->kv_len, c->pend_feat, c->pend_id,
                                               c->feat, c->feat_h, c->cur_id, c->keys, c->key_stride, (const bf16*)c->embed,
                                               V, c->xe_h, c->id_flag, st));

@@ -146,7 +146,7 @@ struct CuSeqlens {
 // weights streamed by TMA into a shared-memory ring, tcgen05.mma with the weights as the M operand
 // (128 rows) and the batch as N (16 columns), accumulators in tensor memory.
 // ---------------------------------------------------------------------------------------------
-#define TC_OP_ROWS 16          // rows of every bf16 operand buffer that the tensor maps cover
+#define TC_OP_ROWS 32          // rows of every bf16 operand buffer that the tensor maps cover
 enum { TCM_W = 0,              // PH_COUNT weight maps, box 64 x 128
        TCM_X_FEAT = PH_COUNT, TCM_X_XQ, TCM_X_ATTN, TCM_X_XM, TCM_X_ACT,   // operand maps, box 64 x 16
        TCM_X_EMB,              // gathered embedding rows, box 64 x 16
@@ -158,7 +158,7 @@ struct TcMaps {
 struct TcArgs {
     ChainPhase ph[PH_COUNT];
     int k, B;
-    int lo;                    // 1: B <= 8, operand rows [B, 2B) carry the bf16 rounding remainders
+    int lo;                    // > 0: operand rows [lo, lo + B) carry the bf16 rounding remainders of rows [0, B)
     int d, qw, kvw, F, V, Hq, Hkv, dh, max_len;
     float eps, scale;
     const bf16 *norm1, *norm2, *bqkv;
@@ -200,6 +200,7 @@ cudaError_t launch_tc_setup(const SlotList& sl, int k, int d, int lo, int* d_slo
                             int* cur_id, u64* keys, int key_stride, const bf16* embed, int vocab, bf16* xe_h,
                             int* id_flag, cudaStream_t st);
 int tc_barriers_per_step();
+int tc_lo_offset(int B);
 
 // ---------------------------------------------------------------------------------------------
 // Small kernels: state set-up, prefill bookkeeping, verification, layout changes, taps.

@@ -44,10 +44,19 @@
 #include "attn_mma.cuh"
 
 #define TC_THREADS 256
-#define TC_STAGES 12
 #define TC_BK 64
 #define TC_TM 128
-#define TC_TN 16
+// Batch columns of one MMA.  32: columns [0,16) take the activations rounded to bf16, columns [16,32) their
+// rounding remainders, for every batch size (an MMA of this shape costs the same for 16 and for 32 columns).
+// 16: the remainders use the unused columns [B, 2B), which exist only for B <= 8.
+#ifndef TC_TN
+#define TC_TN 32
+#endif
+#if TC_TN == 32
+#define TC_STAGES 11
+#else
+#define TC_STAGES 12
+#endif
 #define TC_A_BYTES (TC_TM * TC_BK * 2)
 #define TC_B_BYTES (TC_TN * TC_BK * 2)
 #define TC_ATT_FIRST 4               // first warp that runs the attention
@@ -55,7 +64,7 @@
 #define TC_BAR_ATT 2
 #define TC_EPI_THREADS 128
 #define TC_BAR_EPI 3
-#define TC_TMEM_COLS 32
+#define TC_TMEM_COLS (2 * TC_TN)
 
 // instruction descriptor of tcgen05.mma kind::f16: fp32 accumulate, bf16 x bf16, both K-major, N=16, M=128
 #define TC_IDESC ((1u << 4) | (1u << 7) | (1u << 10) | ((TC_TN >> 3) << 17) | ((TC_TM >> 4) << 24))
@@ -158,17 +167,30 @@ __device__ __forceinline__ u64 tc_smem_desc(uint32_t addr) {
     const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
     return ((u64)hi << 32) | lo;
 }
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
-    uint32_t r[16];
+__device__ __forceinline__ void tc_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
           "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr)
         : "memory");
+}
+// This thread's row of an accumulator: batch columns [0,16) plus the remainder columns that go with them
+// (lo_off columns further on; 0 = none), added here so that everything downstream sees 16 values.
+__device__ __forceinline__ void tc_ld_acc(uint32_t taddr, float (&v)[16], int lo_off) {
+    uint32_t r[16];
+    tc_ld16_issue(taddr, r);
+#if TC_TN == 32
+    uint32_t q[16];
+    tc_ld16_issue(taddr + 16, q);
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]) + (lo_off ? __uint_as_float(q[i]) : 0.f);
+#else
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]) + ((lo_off && i + lo_off < 16) ? __uint_as_float(r[(i + lo_off) & 15]) : 0.f);
+#endif
 }
 __device__ __forceinline__ u64 ld_acquire_u64(const u64* p) {
     u64 v;
@@ -740,13 +762,10 @@ __device__ void epi_output(const TcArgs& a, TcCtl* ctl, int p, int s, int tile, 
     const int row = tile * TC_TM + w4 * 32 + lane;
     const bool rok = row < N;
     const int B = a.B;
-    const int lo_rows = a.lo ? B : 0;
+    const int lo_rows = a.lo;
     float val[16];
 #pragma unroll
-    for (int b = 0; b < 16; ++b) val[b] = 0.f;
-#pragma unroll
-    for (int b = 0; b < 16; ++b)
-        if (b < B) val[b] = v[b] + ((a.lo && b + B < 16) ? v[(b + B) & 15] : 0.f);
+    for (int b = 0; b < 16; ++b) val[b] = b < B ? v[b] : 0.f;
 
     if (p == PH_FC || p == PH_O) {
         float* outf = p == PH_FC ? a.u : a.y;
@@ -932,7 +951,7 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
         wait_mbar(saddr(&ctl->tfull[acc]), (seg_cnt >> 1) & 1u, ctl, a.error_flag, 6);
         tc_fence_after();
         float v[16];
-        tc_ld16(ctl->tmem_base + ((uint32_t)(w4 * 32) << 16) + acc * TC_TN, v);
+        tc_ld_acc(ctl->tmem_base + ((uint32_t)(w4 * 32) << 16) + acc * TC_TN, v, a.lo);
         tc_fence_before();
         mbar_arrive(saddr(&ctl->tempty[acc]));
         ++seg_cnt;
@@ -1073,7 +1092,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
         aw.qkv = a.qkv; aw.ld = a.qw + 2 * a.kvw; aw.Kc = (bf16*)a.Kc; aw.Vc = (bf16*)a.Vc; aw.slots = a.slots;
         aw.pos0 = a.pos0; aw.step = 0; aw.rope_tab = a.rope_tab; aw.Hq = a.Hq; aw.Hkv = a.Hkv; aw.max_len = a.max_len;
         aw.B = a.B; aw.scale = a.scale; aw.part_acc = a.part_acc; aw.part_ml = a.part_ml; aw.nslot = a.attn_nslot;
-        aw.counters = a.counters; aw.attn = a.attn; aw.attn_h = a.attn_h; aw.lo_rows = a.lo ? a.B : 0;
+        aw.counters = a.counters; aw.attn = a.attn; aw.attn_h = a.attn_h; aw.lo_rows = a.lo;
         // ring items of this CTA per step, and those before the attention items of step 0
         unsigned items_step = ai.total, items_before = 0;
         for (int p = 0; p < PH_COUNT; ++p) {
@@ -1132,9 +1151,9 @@ __global__ void tc_setup_kernel(SlotList sl, int k, int d, int lo, int* d_slots,
                                 u64* keys, int key_stride, const bf16* embed, int vocab, bf16* xe_h, int* id_flag) {
     const int b = blockIdx.x;
     if (b >= sl.n) {
-        // Rows of the embedding operand beyond the batch: the tiled copy always brings all 16 rows, and for B <= 8
-        // accumulator columns [B, 2B) are added to columns [0, B) as rounding remainders (an embedding row is exact
-        // in bf16, so its remainder is zero).  An earlier, larger batch may have left rows here.
+        // Rows of the embedding operand beyond the batch: the tiled copy always brings all rows, and the accumulator
+        // columns of the remainder rows are added to those of the batch rows (an embedding row is exact in bf16, so
+        // its remainder is zero).  An earlier, larger batch may have left rows here.
         for (int i = threadIdx.x; i < (d >> 3); i += blockDim.x)
             ((uint4*)(xe_h + (long long)b * d))[i] = make_uint4(0u, 0u, 0u, 0u);
         return;
@@ -1153,7 +1172,7 @@ __global__ void tc_setup_kernel(SlotList sl, int k, int d, int lo, int* d_slots,
         feat[(long long)b * d + i] = v;
         const bf16 hi = __float2bfloat16_rn(v);
         feat_h[(long long)b * d + i] = hi;
-        if (lo) feat_h[(long long)(b + sl.n) * d + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
+        if (lo) feat_h[(long long)(b + lo) * d + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
     }
     // embedding row of the pending token: the fusion FC's embedding operand of step 0
     const int id = checked_token(pend_id[slot], vocab, id_flag);
@@ -1218,6 +1237,16 @@ int tc_max_tiles(const ChainPhase* ph) {
 }
 
 int tc_barriers_per_step() { return TC_BARS_PER_STEP; }
+
+// Row offset of the rounding remainders in the operand buffers for a batch of B (0: none are kept).
+int tc_lo_offset(int B) {
+#if TC_TN == 32
+    (void)B;
+    return 16;
+#else
+    return B <= 8 ? B : 0;
+#endif
+}
 
 cudaError_t tc_build_maps(TcMaps* maps, const ChainPhase* ph, int d, int qw, int F,
                           const bf16* feat_h, const bf16* xq_h, const bf16* attn_h, const bf16* xm_h,
