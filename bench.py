@@ -380,6 +380,78 @@ def time_workload(wl, steps: int, warmup: int, rank: int, local_rank: int, world
             "verify_matches_planted": ok_planted}
 
 
+PHASES = ("gather", "fc", "qkv", "attention", "o_proj", "gate_up", "down", "lm_head")
+
+
+def phase_breakdown(wl, weights: WeightCache, reps: int = 20):
+    """Where a draft step of the tensor-core chain kernel goes: the kernel's own time stamps (option
+    HIVIS_OPT_PHASE_TIMES), `reps` recorded launches, medians over launches.  Per phase: its cost (last arrival on
+    the previous grid barrier -> last arrival on its own), the spread of the arrivals, how long after the previous
+    barrier completed the operand producers got going, and the tail after the last accumulator was complete."""
+    import torch
+    from hivis_inputs.device import to_dev
+    from paper_2509_23928_b200 import Drafter
+    ids, hidden, cu = hi.make_prompt(wl)
+    resid = hi.make_residuals(wl)
+    lens = np.diff(cu)
+    B, k = wl.batch, wl.k
+    dr = Drafter(wl.dims, weights.get(wl), max_batch=B, max_len=int(lens.max()) + k + 8, max_k=max(k, 8))
+    d_resid = to_dev(resid, wl.dims.dtype)
+    dr.prefill(torch.from_numpy(ids).cuda(), to_dev(hidden, wl.dims.dtype), [int(x) for x in cu], resid0=d_resid[0])
+    out_ids = torch.empty((B, k), dtype=torch.int32, device="cuda")
+
+    def restore():
+        for b in range(B):
+            dr.set_kv_len(b, int(lens[b]) - 1, restore_pending=True)
+
+    for _ in range(5):
+        dr.draft(B, k, d_resid, out_ids=out_ids); restore()
+    dr.record_phase_times(True)
+    cost, spread, start, tail, late = [], [], [], [], np.zeros(0)
+    for _ in range(reps):
+        dr.draft(B, k, d_resid, out_ids=out_ids)
+        T = dr.phase_times().astype(np.float64) / 1e3        # [k, events, grid] in us; 0 = no event
+        restore()
+        T[T == 0] = np.nan
+        arr = T[:, :8, :].reshape(k * 8, -1)                 # arrivals in barrier order
+        done = np.nanmax(arr, axis=1)                        # completion of every barrier
+        prev = np.concatenate([[np.nan], done[:-1]])
+        cost.append((done - prev).reshape(k, 8))
+        spread.append((done - np.nanmin(arr, axis=1)).reshape(k, 8))
+        gemm_bar = np.array([1, 2, 4, 5, 6, 7])              # barrier index of the six GEMM phases
+        st = np.full((k, 8), np.nan); tl = np.full((k, 8), np.nan)
+        for s in range(k):
+            for j, e in enumerate(gemm_bar):
+                before = prev[s * 8 + e]
+                st[s, e] = np.nanmedian(T[s, 8 + j]) - before          # operand producers under way
+                tl[s, e] = np.nanmedian(T[s, e] - T[s, 14 + j])        # last accumulator -> arrival
+            st[s, 3] = np.nanmedian(T[s, 20]) - prev[s * 8 + 3]
+        start.append(st); tail.append(tl)
+        lateness = arr - np.nanmin(arr, axis=1, keepdims=True)          # per barrier and CTA
+        late = lateness if late.size == 0 else late + lateness
+    dr.record_phase_times(False)
+    dr.close()
+    med = lambda xs: np.nanmedian(np.stack(xs), axis=0)
+    cost, spread, start, tail = med(cost), med(spread), med(start), med(tail)
+    steps = slice(1, None) if k > 1 else slice(0, None)      # step 0 has no previous barrier for its gather
+    out = {"workload": wl.name, "launches": reps, "unit": "us", "per_phase": {}}
+    for e, name in enumerate(PHASES):
+        out["per_phase"][name] = {"cost": round(float(np.nanmean(cost[steps, e])), 2),
+                                  "arrival_spread": round(float(np.nanmean(spread[steps, e])), 2),
+                                  "input_wait_passed_after": None if np.isnan(start[steps, e]).all() else round(float(np.nanmean(start[steps, e])), 2),
+                                  "tail_after_last_accumulator": None if np.isnan(tail[steps, e]).all() else round(float(np.nanmean(tail[steps, e])), 2)}
+    out["step_us"] = round(float(sum(v["cost"] for v in out["per_phase"].values())), 2)
+    # are the same CTAs late in every phase?  mean lateness per CTA over the GEMM barriers of all steps and launches
+    gemm_rows = [s * 8 + e for s in range(k) for e in (1, 2, 4, 5, 6, 7)]
+    per_cta = np.nanmean(late[gemm_rows], axis=0) / reps
+    order = np.argsort(-per_cta)
+    out["cta_lateness"] = {"mean": round(float(np.nanmean(per_cta)), 2), "max": round(float(np.nanmax(per_cta)), 2),
+                           "latest_ctas": [int(c) for c in order[:12]],
+                           "their_lateness": [round(float(per_cta[c]), 2) for c in order[:12]],
+                           "earliest_ctas": [int(c) for c in order[-6:]]}
+    return out
+
+
 def stub_replica(rank: int) -> dict:
     """Stands in for the device work when HIVIS_BENCH_STUB=1 (CPU test of the launch path only): fixed fake
     times, rank 1 slower.  The line it leads to is marked as a stub and carries no measurement."""
@@ -395,6 +467,8 @@ def main():
     ap.add_argument("--workload", default=None, help="time this workload only (default: batch 1, then batch 16)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--phase-times", action="store_true",
+                    help="print where a draft step of the tensor-core chain kernel goes (its own time stamps) and exit")
     args = ap.parse_args()
     if args.gpus < 1:
         ap.error("--gpus must be at least 1")
@@ -446,6 +520,9 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     wl = replica_workload(wl, rank, world)                 # independent replicas, same shapes
     weights = WeightCache()
+    if args.phase_times:
+        print(json.dumps(phase_breakdown(hi.workload(args.workload or BATCH16), weights)))
+        return
     res = time_workload(wl, args.steps, args.warmup, rank, local_rank, world, dist, weights, not args.no_e2e)
 
     extra = {}

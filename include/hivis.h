@@ -192,9 +192,30 @@ int hivis_debug_tap(hivis_ctx* ctx, int which, float* out, void* stream);
  * reports and returns in an orderly way.
  * HIVIS_OPT_DEBUG_MISS_BARRIER (test aid): 1 makes the grid barriers of the NEXT hivis_draft call
  * impossible to complete, so that every wait runs into its limit: hivis_status then returns
- * HIVIS_ERR_TIMEOUT and the context is usable again.  Nothing faults or hangs.                          */
-enum { HIVIS_OPT_CHAIN_KERNEL = 0, HIVIS_OPT_TC_KERNEL = 1, HIVIS_OPT_WAIT_LIMIT_US = 2, HIVIS_OPT_DEBUG_MISS_BARRIER = 3 };
+ * HIVIS_ERR_TIMEOUT and the context is usable again.  Nothing faults or hangs.
+ * HIVIS_OPT_PHASE_TIMES (default 0): 1 makes the tensor-core chain kernel write a time stamp per CTA at the
+ * events listed under hivis_read_phase_times (a store per event; off, the kernel only tests a pointer).    */
+enum { HIVIS_OPT_CHAIN_KERNEL = 0, HIVIS_OPT_TC_KERNEL = 1, HIVIS_OPT_WAIT_LIMIT_US = 2, HIVIS_OPT_DEBUG_MISS_BARRIER = 3,
+       HIVIS_OPT_PHASE_TIMES = 4 };
 int hivis_set_option(hivis_ctx* ctx, int option, int value);
+
+/* Where the time of a draft step goes: synchronises `stream` and copies the time stamps of the LAST hivis_draft
+ * that ran the tensor-core chain kernel with HIVIS_OPT_PHASE_TIMES on.  out_host[(s * HIVIS_PHASE_EVENTS + e) *
+ * grid + cta] = time in ns (the GPU's global timer) of event e of draft step s on CTA cta; 0 where the event did
+ * not occur (a CTA without work in a phase).  Events:
+ *   0..7   the CTA's arrival on the grid barrier after: embedding gather, fusion FC, QKV, attention, O, gate/up,
+ *          down, LM head (the time from the last arrival on one barrier to the last arrival on the next is what
+ *          that phase costs);
+ *   8..13  the CTA's operand producer got past its wait for the phase's input (FC, QKV, O, gate/up, down, LM head);
+ *   14..19 the last accumulator of the CTA's range in that phase was complete (what follows is the phase's tail:
+ *          partial sums, output stage, barrier);
+ *   20     the CTA's attention warps got past their wait for the QKV phase.
+ * k_host, grid_host: draft steps and CTAs recorded.  capacity: entries out_host can take; with less than
+ * k * HIVIS_PHASE_EVENTS * grid the call fills k_host and grid_host and returns HIVIS_ERR_CAPACITY.
+ * Errors: ARG, STATE (nothing recorded), CAPACITY, CUDA.                                                    */
+#define HIVIS_PHASE_EVENTS 24
+int hivis_read_phase_times(hivis_ctx* ctx, uint64_t* out_host, long long capacity, int* k_host, int* grid_host,
+                           void* stream);
 
 /* Synchronises `stream` and reports what the kernels since the last call recorded:
  * HIVIS_ERR_TIMEOUT - a kernel gave up on a bounded device-side wait (the outputs of that call

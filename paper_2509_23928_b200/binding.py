@@ -17,11 +17,13 @@ ERRORS = {0: "OK", -1: "ARG", -2: "SHAPE", -3: "DTYPE", -4: "STATE", -5: "CAPACI
 EXPORTS = ("hivis_init", "hivis_destroy", "hivis_prefill", "hivis_draft", "hivis_verify", "hivis_reset",
            "hivis_get_kv_len", "hivis_set_kv_len", "hivis_read_kv", "hivis_debug_tap", "hivis_step_bytes",
            "hivis_launch_count", "hivis_last_error", "hivis_profile_begin", "hivis_profile_end", "hivis_set_option",
-           "hivis_status", "hivis_verify_noalloc")
+           "hivis_status", "hivis_verify_noalloc", "hivis_read_phase_times")
 HIVIS_OPT_CHAIN_KERNEL = 0
 HIVIS_OPT_TC_KERNEL = 1
 HIVIS_OPT_WAIT_LIMIT_US = 2
 HIVIS_OPT_DEBUG_MISS_BARRIER = 3
+HIVIS_OPT_PHASE_TIMES = 4
+HIVIS_PHASE_EVENTS = 24
 PROFILE_CLASSES = ("fuse_fc", "qkv", "attention", "o_proj", "gate_up", "down", "lm_head_argmax", "setup_finish",
                    "draft_chain")
 
@@ -74,6 +76,7 @@ def _load() -> C.CDLL:
     L.hivis_profile_begin.argtypes = [vp]
     L.hivis_profile_end.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int64)]
     L.hivis_verify_noalloc.argtypes = [i32, i32, i32, vp, vp, i32, vp, vp, vp, vp, vp]
+    L.hivis_read_phase_times.argtypes = [vp, vp, C.c_longlong, ip, ip, vp]
     L.hivis_last_error.argtypes = [vp]
     L.hivis_last_error.restype = C.c_char_p
     for n in EXPORTS:
@@ -201,6 +204,19 @@ def hivis_profile_end(ctx):
     return {name: (float(ms[i]), int(n[i])) for i, name in enumerate(PROFILE_CLASSES)}
 
 
+def hivis_read_phase_times(ctx, stream=None):
+    """-> uint64 array [k, HIVIS_PHASE_EVENTS, grid] of the last recorded tensor-core chain launch (ns; 0 = no event)."""
+    import numpy as np
+    k, g = C.c_int(), C.c_int()
+    rc = lib.hivis_read_phase_times(ctx, None, 0, C.byref(k), C.byref(g), _stream(stream))
+    if rc != -5:
+        _check(rc, ctx)
+    out = np.zeros((k.value, HIVIS_PHASE_EVENTS, g.value), dtype=np.uint64)
+    _check(lib.hivis_read_phase_times(ctx, out.ctypes.data_as(C.c_void_p), out.size, C.byref(k), C.byref(g),
+                                      _stream(stream)), ctx)
+    return out
+
+
 def hivis_launch_count(ctx) -> int:
     return int(lib.hivis_launch_count(ctx))
 
@@ -298,6 +314,12 @@ class Drafter:
     def miss_next_barrier(self):
         """Test aid: the grid barriers of the next draft cannot complete, so its waits run out."""
         hivis_set_option(self.ctx, HIVIS_OPT_DEBUG_MISS_BARRIER, 1)
+
+    def record_phase_times(self, on: bool = True):
+        hivis_set_option(self.ctx, HIVIS_OPT_PHASE_TIMES, 1 if on else 0)
+
+    def phase_times(self):
+        return hivis_read_phase_times(self.ctx)
 
     def status(self):
         hivis_status(self.ctx)

@@ -49,6 +49,9 @@ struct hivis_ctx {
     long long wait_cycles;        // option HIVIS_OPT_WAIT_LIMIT_US, in cycles
     bool debug_skew;              // option HIVIS_OPT_DEBUG_MISS_BARRIER: the next draft's grid barriers cannot complete
     int opt_tc;                   // option HIVIS_OPT_TC_KERNEL: 0 off, 1 for two or more sequences, 2 always
+    bool opt_phase_times;         // option HIVIS_OPT_PHASE_TIMES
+    u64* phase_t;                 // [HIVIS_MAX_K][HIVIS_PHASE_EVENTS][num_sms]
+    int phase_k;                  // draft steps of the last recorded launch (0: none)
     TcMaps tc_maps;
     float* tc_partial;
     int* tile_ctr;
@@ -256,6 +259,9 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
     c->debug_skew = false;
     c->tc_ok = false;
     c->tc_partial = nullptr;
+    c->opt_phase_times = false;
+    c->phase_t = nullptr;
+    c->phase_k = 0;
     c->tile_ctr = nullptr;
     c->tc_tiles = 0;
     c->bar_count_host = 0;
@@ -369,7 +375,8 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
         ChainArgs ca;
         fill_chain_args(c, &ca);
         c->tc_tiles = tc_max_tiles(ca.ph);
-        bool ok2 = dalloc(c, &c->tc_partial, (size_t)c->num_sms * 2 * 16 * 128) && dalloc(c, &c->tile_ctr, c->tc_tiles);
+        bool ok2 = dalloc(c, &c->tc_partial, (size_t)c->num_sms * 2 * 16 * 128) && dalloc(c, &c->tile_ctr, c->tc_tiles) &&
+                   dalloc(c, &c->phase_t, (size_t)HIVIS_MAX_K * HIVIS_PHASE_EVENTS * c->num_sms);
         if (ok2) ok2 = cudaMemsetAsync(c->tile_ctr, 0, c->tc_tiles * sizeof(int), st) == cudaSuccess;
         if (ok2)
             ok2 = tc_build_maps(&c->tc_maps, ca.ph, cfg->d, c->qw, cfg->ffn, c->feat_h, c->xq, c->attn_h, c->xm, c->act_h,
@@ -634,6 +641,12 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
         a.attn_nslot = c->nsplit_cap;
         a.bar_counter = c->bar_counter; a.bar_base = c->bar_count_host + (c->debug_skew ? (1ull << 40) : 0ull);
         a.wait_cycles = c->wait_cycles; a.error_flag = c->error_flag; a.id_flag = c->id_flag;
+        a.phase_t = nullptr;
+        if (c->opt_phase_times) {
+            CK(c, cudaMemsetAsync(c->phase_t, 0, (size_t)k * HIVIS_PHASE_EVENTS * c->num_sms * sizeof(u64), st));
+            a.phase_t = c->phase_t;
+            c->phase_k = k;
+        }
         c->debug_skew = false;
         CKP(c, CLS_CHAIN, st, launch_tc_chain(c->tc_maps, a, c->num_sms, st));
         c->bar_count_host += (u64)c->num_sms * (u64)(tc_barriers_per_step() * k);
@@ -848,6 +861,10 @@ int hivis_set_option(hivis_ctx* c, int option, int value) {
         c->debug_skew = value != 0;
         return HIVIS_OK;
     }
+    if (option == HIVIS_OPT_PHASE_TIMES) {
+        c->opt_phase_times = value != 0;
+        return HIVIS_OK;
+    }
     return fail(c, HIVIS_ERR_ARG, "unknown option %d", option);
 }
 
@@ -872,6 +889,21 @@ int hivis_status(hivis_ctx* c, void* stream) {
     CK(c, cudaStreamSynchronize(st));
     c->bar_count_host = 0;
     return fail(c, HIVIS_ERR_TIMEOUT, "a device-side wait ran out (code %d); results of that call are invalid", flag);
+}
+
+int hivis_read_phase_times(hivis_ctx* c, uint64_t* out_host, long long capacity, int* k_host, int* grid_host,
+                           void* stream) {
+    if (!c) return HIVIS_ERR_ARG;
+    if (!k_host || !grid_host) return fail(c, HIVIS_ERR_ARG, "null argument");
+    if (c->phase_k == 0 || !c->phase_t) return fail(c, HIVIS_ERR_STATE, "no draft has recorded phase times");
+    *k_host = c->phase_k;
+    *grid_host = c->num_sms;
+    const long long n = (long long)c->phase_k * HIVIS_PHASE_EVENTS * c->num_sms;
+    if (!out_host || capacity < n) return fail(c, HIVIS_ERR_CAPACITY, "phase times need room for %lld entries", n);
+    cudaStream_t st = (cudaStream_t)stream;
+    CK(c, cudaMemcpyAsync(out_host, c->phase_t, (size_t)n * sizeof(u64), cudaMemcpyDeviceToHost, st));
+    CK(c, cudaStreamSynchronize(st));
+    return HIVIS_OK;
 }
 
 int hivis_profile_begin(hivis_ctx* c) {

@@ -210,6 +210,13 @@ __device__ __forceinline__ int ld_relaxed_int(const int* p) {
     asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
+// Optional time stamps (HIVIS_OPT_PHASE_TIMES): event e of step s on this CTA, in nanoseconds of the GPU's global timer.
+__device__ __forceinline__ void phase_stamp(const TcArgs& a, int s, int e, int cta, int G) {
+    if (a.phase_t == nullptr) return;
+    u64 t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    a.phase_t[((long long)s * HIVIS_PHASE_EVENTS + e) * G + cta] = t;
+}
 __device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 
 // ---- bounded waits -------------------------------------------------------------------------------
@@ -563,6 +570,7 @@ __device__ void tc_producer_x(const TcParams& P, TcCtl* ctl, uint32_t smemB, int
                 // other CTAs wrote the operand through the generic proxy; TMA reads through the async proxy
                 fence_proxy_async_global();
             }
+            phase_stamp(a, c.step, 8 + c.p, cta, G);
         }
         const bool emb = c.p == PH_FC && c.kb >= dkb;
         if (emb && gathered_step != c.step) {
@@ -621,6 +629,7 @@ __device__ void tc_gather(const TcParams& P, TcCtl* ctl, int s, int cta, int G, 
     }
     __syncwarp();
     if (lane == 0) {
+        phase_stamp(a, s, TC_SEQ_GATHER, cta, G);
         red_release_add_u64(a.bar_counter, 1ull);
     }
     __syncwarp();
@@ -949,6 +958,7 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
         }
         const unsigned acc = seg_cnt & 1u;
         wait_mbar(saddr(&ctl->tfull[acc]), (seg_cnt >> 1) & 1u, ctl, a.error_flag, 6);
+        if (etid == 0 && idx + n == hi) phase_stamp(a, s, 14 + p, cta, G);
         tc_fence_after();
         float v[16];
         tc_ld_acc(ctl->tmem_base + ((uint32_t)(w4 * 32) << 16) + acc * TC_TN, v, a.lo);
@@ -1024,6 +1034,7 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
         const int need = p == PH_FC ? s * TC_BARS_PER_STEP + TC_SEQ_GATHER : need_seq(s, p);
         if ((lo == hi || p == PH_FC) && need >= 0)
             wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(need + 1), ctl, a.error_flag, 8);
+        phase_stamp(a, s, phase_seq(p), cta, G);
         red_release_add_u64(a.bar_counter, 1ull);
     }
     // Without work in the phase nothing but the wait above tells this CTA that the earlier phases are complete:
@@ -1116,6 +1127,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
             if (atid < 0) continue;
             if (atid == 0)
                 wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(s * TC_BARS_PER_STEP + TC_SEQ_ATTN), ctl, a.error_flag, 7);
+            if (atid == 0) phase_stamp(a, s, 20, cta, G);
             named_sync(TC_BAR_ATT, TC_ATT_WARPS * 32);
             if (!poisoned(ctl)) {
                 aw.step = s;
@@ -1126,6 +1138,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
             }
             named_sync(TC_BAR_ATT, TC_ATT_WARPS * 32);
             if (atid == 0) {
+                phase_stamp(a, s, TC_SEQ_ATTN, cta, G);
                 red_release_add_u64(a.bar_counter, 1ull);
             }
             if (is_epi) {
