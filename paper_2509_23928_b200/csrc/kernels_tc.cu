@@ -226,8 +226,8 @@ __device__ __forceinline__ void poison(TcCtl* ctl, int* error_flag, int code) {
     *(volatile int*)&ctl->abort_flag = 1;
 }
 __device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, TcCtl* ctl, int* error_flag, int code) {
+    if (mbar_try(bar, parity)) return true;         // the usual case costs one instruction; a completed phase is safe to use
     if (poisoned(ctl)) return false;
-    if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
     unsigned it = 0;
     while (!mbar_try(bar, parity)) {
