@@ -524,8 +524,8 @@ __device__ void tc_producer_w(const TcParams& P, TcCtl* ctl, uint32_t smemA, int
             publish = TC_STAGES;
         }
         if (!ok) break;
+        // (after a give-up nobody hands stages back, so the wait below ends the loop: no separate look at the flag)
         if (round > 0 && !wait_mbar(saddr(&ctl->empty[slot]), (round - 1) & 1u, ctl, a.error_flag, 3)) break;
-        if (poisoned(ctl)) break;
         const uint32_t bar = saddr(&ctl->full[slot]);
         mbar_expect_tx(bar, TC_A_BYTES + TC_B_BYTES);
         tma_load_2d(smemA + slot * TC_A_BYTES, &P.maps.m[TCM_W + c.p], c.kb * TC_BK, c.tile * TC_TM, bar, pol_w);
@@ -581,7 +581,6 @@ __device__ void tc_producer_x(const TcParams& P, TcCtl* ctl, uint32_t smemB, int
             gathered_step = c.step;
         }
         if (round > 0 && !wait_mbar(saddr(&ctl->empty[slot]), (round - 1) & 1u, ctl, a.error_flag, 10)) break;
-        if (poisoned(ctl)) break;
         const uint32_t bar = saddr(&ctl->full[slot]);
         const uint32_t dst = smemB + slot * TC_B_BYTES;
         if (emb) tma_load_2d(dst, &P.maps.m[TCM_X_EMB], (c.kb - dkb) * TC_BK, 0, bar, pol_x);
