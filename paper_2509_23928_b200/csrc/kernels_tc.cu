@@ -456,16 +456,27 @@ __device__ bool tc_issue_attention(const TcParams& P, TcCtl* ctl, uint32_t smemA
         for (int w = 0; w < TC_ATT_WARPS; ++w) {
             if (cur[w].left == 0) continue;
             any = true;
-            if (round > 0 && !wait_mbar(saddr(&ctl->empty[slot]), (round - 1) & 1u, ctl, a.error_flag, 14)) return false;
-            if (poisoned(ctl)) return false;
+            // everything the copies need is worked out before the wait for the stage: what follows the wait is on the
+            // path of every item (after a give-up nobody hands stages back, so the wait itself ends the loop)
+            const bool tail_item = cur[w].j == cur[w].nb - 1;
+            const int kvh = cur[w].hg * GQ / Gh;
+            const uint32_t dst = smemA + slot * TC_A_BYTES;
             const uint32_t bar = saddr(&ctl->full[slot]);
-            if (cur[w].j == cur[w].nb - 1) {
+            int row0 = 0;
+            uint32_t bytes = 0;
+            long long off = 0;
+            if constexpr (AttSel<GQ>::mma) {
+                row0 = (cur[w].slot * a.Hkv + kvh) * a.max_len + 32 * cur[w].j;
+            } else if (!tail_item) {
+                const int left_rows = cur[w].rows - 32 * cur[w].j;
+                bytes = (uint32_t)(left_rows < 32 ? left_rows : 32) * (DH * 2);
+                off = (((long long)__ldg(a.slots + cur[w].b) * a.Hkv + kvh) * (long long)a.max_len + 32 * cur[w].j) * DH;
+            }
+            if (round > 0 && !wait_mbar(saddr(&ctl->empty[slot]), (round - 1) & 1u, ctl, a.error_flag, 14)) return false;
+            if (tail_item) {
                 mbar_arrive(bar);
             } else {
-                const int kvh = cur[w].hg * GQ / Gh;
-                const uint32_t dst = smemA + slot * TC_A_BYTES;
                 if constexpr (AttSel<GQ>::mma) {
-                    const int row0 = (cur[w].slot * a.Hkv + kvh) * a.max_len + 32 * cur[w].j;
                     mbar_expect_tx(bar, 2 * 32 * DH * 2);
 #pragma unroll
                     for (int h = 0; h < DH / 64; ++h) {
@@ -473,10 +484,6 @@ __device__ bool tc_issue_attention(const TcParams& P, TcCtl* ctl, uint32_t smemA
                         tma_load_2d(dst + 32 * DH * 2 + h * 4096, &P.maps.m[TCM_V], 64 * h, row0, bar, pol);
                     }
                 } else {
-                    const int left_rows = cur[w].rows - 32 * cur[w].j;
-                    const uint32_t bytes = (uint32_t)(left_rows < 32 ? left_rows : 32) * (DH * 2);
-                    const long long off =
-                        (((long long)__ldg(a.slots + cur[w].b) * a.Hkv + kvh) * (long long)a.max_len + 32 * cur[w].j) * DH;
                     mbar_expect_tx(bar, 2 * bytes);
                     bulk_load(dst, (const bf16*)a.Kc + off, bytes, bar);
                     bulk_load(dst + 32 * DH * 2, (const bf16*)a.Vc + off, bytes, bar);
