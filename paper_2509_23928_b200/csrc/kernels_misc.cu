@@ -151,7 +151,7 @@ cudaError_t launch_kv_append(int dtype, const float* kv, int P, const int* slot_
 // ------------------------------------------------------------------------------------------
 // greedy verification in one launch: row argmax over [B][k+1][V], accept length, next token, rollback
 // ------------------------------------------------------------------------------------------
-#define VERIFY_CHUNK 8192   // logits per CTA
+#define VERIFY_CHUNK 2048   // logits per CTA: one 16-byte load per thread for bf16 logits
 
 // One CTA per (chunk of a row, row, sequence).  Every CTA folds its chunk into the row's packed argmax key
 // (integer max: lowest index among equal values, independent of arrival order) and counts itself on the

@@ -6,16 +6,21 @@
 //                        ring with TMA (cp.async.bulk.tensor, 128-byte swizzle, mbarrier complete_tx).
 //                        Weight tiles do not depend on activations, so their loads run ahead through phase
 //                        and step boundaries, limited only by the ring.
-//   warp 2 (one thread)  operand producer: the matching batch-operand tiles (16 rows x 64 k, 2 KB) in the
+//   warp 2 (one thread)  operand producer: the matching batch-operand tiles (32 rows x 64 k, 4 KB) in the
 //                        same order; the first tile of a phase waits for the grid barrier before it.
-//   warp 3               embedding gather: once a step's tokens are known, copies their embedding rows into
-//                        the dense operand buffer of the fusion FC's embedding half (a barrier of its own).
-//   warp 1 (one thread)  issues tcgen05.mma (M = 128 weight rows, N = 16 batch columns, K = 16, four per
-//                        stage), accumulating in tensor memory (two 16-column accumulators, so the next
+//   warp 3               no role.
+//   warp 1 (one thread)  issues tcgen05.mma (M = 128 weight rows, N = 32 batch columns, K = 16, four per
+//                        stage), accumulating in tensor memory (two 32-column accumulators, so the next
 //                        tile's MMAs overlap the previous tile's epilogue); tcgen05.commit frees stages.
+//   The three single threads are the pace of the whole kernel: a stage's round trip (handed back -> copy
+//   issued -> landed -> MMAs issued -> handed back) bounds the bytes in flight, so their loops hold nothing
+//   that is not needed per item (one shared-memory load more per wait cost 2-4 % of a draft step).
 //   warps 4-7            epilogue: tcgen05.ld (one weight row per thread, 16 batch values), then the fused
 //                        output stage of the phase (residuals, RMSNorm statistics and gains, RoPE-free
 //                        QKV bias, SiLU*up, LM-head argmax keys) and the bf16 operand of the next phase.
+//   warps 4-7            at the start of a step: embedding gather - once the step's tokens are known, their
+//                        embedding rows are copied into the dense operand buffer of the fusion FC's embedding
+//                        half (a grid barrier of its own).
 //   warps 4-7            between the QKV and O phases: split-KV attention over the text-only cache (one warp per
 //                        scheduler: a fifth warp sharing a scheduler with another slowed both).  Its K/V
 //                        blocks travel through the same ring: the rows a sequence had when the launch began
@@ -30,9 +35,9 @@
 // range is at least a tile long, the tile at its end is finished from an early look at the counter (the other
 // contributors did their part at the start of the phase).  Nobody waits for anybody inside a phase.
 //
-// Batch operand: activations are rounded to bf16 for the MMA; for B <= 8 the rounding remainder is fed
-// through the unused columns (rows [B, 2B) of every operand buffer) and added in the output stage, which
-// keeps about 16 mantissa bits of the activations.
+// Batch operand: activations are rounded to bf16 for the MMA; the rounding remainder of every activation is
+// fed through 16 more batch columns (rows [16, 32) of every operand buffer) and added in the output stage,
+// which keeps about 16 mantissa bits of the activations for every batch size.
 //
 // Every wait is bounded.  A wait that runs out raises the error flag and poisons the CTA: all roles then
 // run through their remaining schedule without waiting, issuing no further copies or MMAs, so that named
@@ -598,17 +603,18 @@ __device__ void tc_producer_x(const TcParams& P, TcCtl* ctl, uint32_t smemB, int
     if (poisoned(ctl)) drain_after_poison();
 }
 
-// Embedding gather of step s (one warp per CTA): once the previous LM head is complete the chosen tokens are
-// known; their embedding rows are copied into the dense operand buffer that the fusion FC reads.  Step 0's rows
-// were copied by the set-up kernel.  Arrives on the gather barrier of the step.
-__device__ void tc_gather(const TcParams& P, TcCtl* ctl, int s, int cta, int G, int lane) {
+// Embedding gather of step s (the four epilogue warps of every CTA, before they turn to the fusion FC): once the
+// previous LM head is complete the chosen tokens are known; their embedding rows are copied into the dense operand
+// buffer that the fusion FC reads.  Step 0's rows were copied by the set-up kernel.  Arrives on the gather barrier
+// of the step.
+__device__ void tc_gather(const TcParams& P, TcCtl* ctl, int s, int cta, int G, int etid) {
     const TcArgs& a = P.a;
     {
         // (cos, sin) of every sequence's new position at this step, for the attention of this step; the two
         // halves of the table alternate between steps, since CTAs still in the previous attention read the other
         const int half = a.dh >> 1;
         float2* tab = a.rope_tab + (long long)(s & 1) * 16 * half;
-        for (int i = cta * 32 + lane; i < a.B * half; i += G * 32) {
+        for (int i = cta * TC_EPI_THREADS + etid; i < a.B * half; i += G * TC_EPI_THREADS) {
             const int b = i / half, f = i - b * half;
             float cs, sn;
             rope_cs(__ldg(a.pos0 + b) + s, a.inv_freq[f], cs, sn);
@@ -616,14 +622,13 @@ __device__ void tc_gather(const TcParams& P, TcCtl* ctl, int s, int cta, int G, 
         }
     }
     if (s > 0) {
-        bool ok = true;
-        if (lane == 0)
-            ok = wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)((s - 1) * TC_BARS_PER_STEP + 8), ctl, a.error_flag, 12);
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        if (ok) {
+        if (etid == 0)
+            wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)((s - 1) * TC_BARS_PER_STEP + 8), ctl, a.error_flag, 12);
+        named_sync(TC_BAR_EPI, TC_EPI_THREADS);
+        if (!poisoned(ctl)) {
             const int upr = a.d >> 3;                    // 16-byte units per row
             const int total = a.B * upr;
-            for (int i = cta * 32 + lane; i < total; i += G * 32) {
+            for (int i = cta * TC_EPI_THREADS + etid; i < total; i += G * TC_EPI_THREADS) {
                 const int b = i / upr, off = i - b * upr;
                 int id = a.forced ? __ldcg(a.forced + (long long)b * a.k + (s - 1))
                                   : key_index(__ldcg(a.keys + (long long)b * a.key_stride + (s - 1)));
@@ -633,12 +638,11 @@ __device__ void tc_gather(const TcParams& P, TcCtl* ctl, int s, int cta, int G, 
             }
         }
     }
-    __syncwarp();
-    if (lane == 0) {
+    named_sync(TC_BAR_EPI, TC_EPI_THREADS);
+    if (etid == 0) {
         phase_stamp(a, s, TC_SEQ_GATHER, cta, G);
         red_release_add_u64(a.bar_counter, 1ull);
     }
-    __syncwarp();
 }
 
 // ---- MMA issuer ----------------------------------------------------------------------------------
@@ -1098,11 +1102,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
     } else if (warp == 2) {
         if (lane == 0) tc_producer_x(P, ctl, smemB, cta, G, ai.total);
         __syncwarp();
-    } else {
-        // warps 4..7: epilogue of every GEMM phase and the attention between the QKV and O phases; warp 3: the
-        // embedding gather
-        const int atid = tid - 32 * TC_ATT_FIRST;        // < 0: not an attention warp
-        const bool is_epi = warp >= 4;
+    } else if (warp >= 4) {
+        // warps 4..7: the embedding gather at the start of a step, the epilogue of every GEMM phase and the attention
+        // between the QKV and O phases
+        // (warp 3 has no role: the epilogue warps must be warps 4..7, since a warp reads the 32 lanes of tensor memory
+        // that its number modulo 4 selects)
+        const int atid = tid - 32 * TC_ATT_FIRST;
+        const bool is_epi = true;
         const int w4 = warp - 4;
         unsigned seg_cnt = 0;
         AttnWArgs aw;
@@ -1124,13 +1130,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
         for (int w = 0; w < TC_ATT_WARPS; ++w) ring.n[w] = ai.n[w];
         for (int s = 0; s < a.k; ++s) {
             if (is_epi) {
+                tc_gather(P, ctl, s, cta, G, atid);
                 tc_epilogue_phase(P, ctl, s, PH_FC, seg_cnt, cta, G, w4, lane);
                 tc_epilogue_phase(P, ctl, s, PH_QKV, seg_cnt, cta, G, w4, lane);
-            } else {
-                tc_gather(P, ctl, s, cta, G, lane);
             }
             // ---- attention: needs every CTA's QKV rows
-            if (atid < 0) continue;
             if (atid == 0)
                 wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(s * TC_BARS_PER_STEP + TC_SEQ_ATTN), ctl, a.error_flag, 7);
             if (atid == 0) phase_stamp(a, s, 20, cta, G);
