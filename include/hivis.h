@@ -153,6 +153,43 @@ int hivis_verify(hivis_ctx* ctx, int B, const int* seq_slots_host, int k,
                  const int32_t* draft_ids, const void* target_logits, int logits_dtype,
                  int32_t* out_accept, int32_t* out_next, int32_t* out_kv_len, void* stream);
 
+/* Tree drafting for ONE sequence (Sec. 2.1: the paper drafts with the dynamic draft tree of EAGLE-2;
+ * "Inference Setup": top-10 expansion, depth 6, the 60 paths of highest cumulative probability kept;
+ * supplementary material, Sec. A: 8 per expansion, depth 4, 30 kept).
+ * Level 0 runs the slot's pending pair at its next cache row P and proposes the `topk` most probable
+ * tokens.  Level l = 1..depth-1 runs the `topk` candidates of depth l with the highest cumulative
+ * log-probability (the frontier) as one batch: input = (layer output of the forward that proposed the
+ * node, the node's token) at position P + l, residual row min(l, n_resid-1), attention over the prefix,
+ * the node's ancestors and itself; each proposes `topk` candidates of depth l + 1, score = parent's score
+ * + log-softmax(logits)[token].  Of all topk + (depth-1)*topk^2 candidates the `keep` with the highest
+ * score are returned in creation order (level by level, parents in frontier order, children by rank), so
+ * a node's parent precedes it.  Equal scores: the candidate created first; equal logits: the lower token.
+ *   out_tokens, out_parents (index into the list, -1 = child of the root) int32 [keep], out_scores fp32
+ *   [keep], out_count int32 [1] = number of nodes written (min(keep, number of candidates)).
+ * The slot's row count does not change until hivis_verify_tree; rows [P, P + 1 + (depth-1)*topk) of the
+ * slot are used for the tree's K/V rows, so that many rows must be free (CAPACITY otherwise).
+ * Limits: 1 <= topk <= HIVIS_TREE_MAX_TOPK, 1 <= depth <= max_k, 1 <= keep <= HIVIS_TREE_MAX_KEEP.
+ * Errors: ARG, STATE (no pending pair), CAPACITY, CUDA.                                              */
+#define HIVIS_TREE_MAX_TOPK 16
+#define HIVIS_TREE_MAX_KEEP 256
+int hivis_draft_tree(hivis_ctx* ctx, int slot, int topk, int depth, int keep, const void* resid, int n_resid,
+                     int32_t* out_tokens, int32_t* out_parents, float* out_scores, int32_t* out_count,
+                     void* stream);
+
+/* Greedy verification of the tree drafted last on the slot, and KV compaction (Sec. 2.1; Algorithm 1,
+ * lines 8-9).  target_logits: [count + 1, vocab] in logits_dtype: row 0 is the target's prediction after
+ * the root token, row 1 + i its prediction after the path that ends in kept node i.  From the root, the
+ * child that carries argmax(row of the current node) is accepted (lowest index on ties) for as long as
+ * there is one.  out_accept[0] = n accepted nodes (0..depth), out_path int32 [depth] = their indices
+ * (-1 beyond n), out_next[0] = argmax(row of the last accepted node): the correction or bonus token.
+ * The slot then holds P + 1 + m rows (also written to out_kv_len, nullable): the root's row and, right
+ * behind it in path order, the K/V rows of the m accepted nodes that were run through the layer (nodes
+ * of the last level were not, like the last token of a chained draft).  Must follow hivis_draft_tree on
+ * the slot.  Errors: ARG, DTYPE, STATE, CUDA.                                                        */
+int hivis_verify_tree(hivis_ctx* ctx, int slot, const void* target_logits, int logits_dtype,
+                      int32_t* out_accept, int32_t* out_path, int32_t* out_next, int32_t* out_kv_len,
+                      void* stream);
+
 /* Forget a sequence: zero rows, no pending pair.                                              */
 int hivis_reset(hivis_ctx* ctx, int slot, void* stream);
 

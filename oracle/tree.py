@@ -56,6 +56,8 @@ class DraftTree:
     root_k: np.ndarray = None     # K/V row of the root position (row P of the cache)
     root_v: np.ndarray = None
     n_cached: int = 0
+    margin: float = np.inf        # smallest gap between neighbours in any ranking that decided the tree's shape or order:
+                                  # an implementation whose scores are off by less than half of it builds the same tree
 
 
 def tree_draft(o, n_cached: int, pend_id: int, pend_hidden, rho, Kc, Vc, topk: int, depth: int, keep: int) -> DraftTree:
@@ -75,11 +77,19 @@ def tree_draft(o, n_cached: int, pend_id: int, pend_hidden, rho, Kc, Vc, topk: i
         g = o.position(feature, int(token), rho[min(level, R - 1)], P + level, kc, vc)
         return g, kc[P + level].copy(), vc[P + level].copy(), log_softmax(lm @ g)
 
+    margin = [np.inf]
+
+    def note_gaps(values_sorted_desc):
+        v = np.asarray(values_sorted_desc, np.float64)
+        if v.size > 1:
+            margin[0] = min(margin[0], float(np.min(v[:-1] - v[1:])))
+
     # candidate list (creation order)
     tok, par, dep, sc = [], [], [], []
     exp_k, exp_v = {}, {}                                   # candidate index -> its K/V row once expanded
     g_root, rk, rv, lp = forward(np.asarray(pend_hidden, o.rt), pend_id, 0, [], [])
     frontier = []                                           # (candidate index, feature to feed with it)
+    note_gaps(lp[top_k(lp, topk + 1)])
     for t in top_k(lp, topk):
         tok.append(int(t)); par.append(-1); dep.append(1); sc.append(float(lp[t]))
         frontier.append((len(tok) - 1, g_root))
@@ -96,13 +106,16 @@ def tree_draft(o, n_cached: int, pend_id: int, pend_hidden, rho, Kc, Vc, topk: i
             anc_v = [rv] + [exp_v[a] for a in chain]
             g, kr, vr, lp = forward(feat, tok[ci], level, anc_k, anc_v)
             exp_k[ci], exp_v[ci] = kr, vr
+            note_gaps(lp[top_k(lp, topk + 1)])
             for t in top_k(lp, topk):
                 tok.append(int(t)); par.append(ci); dep.append(level + 1); sc.append(sc[ci] + float(lp[t]))
                 children.append((len(tok) - 1, g))
         if level + 1 < depth:
+            note_gaps(sorted((sc[c[0]] for c in children), reverse=True)[:topk + 1])
             order = sorted(range(len(children)), key=lambda i: (-sc[children[i][0]], children[i][0]))[:topk]
             frontier = [children[i] for i in sorted(order)]          # frontier kept in creation order
     n_all = len(tok)
+    note_gaps(sorted(sc, reverse=True)[:keep + 1])
     ranked = sorted(range(n_all), key=lambda i: (-sc[i], i))[:min(keep, n_all)]
     kept = sorted(ranked)
     pos = {c: i for i, c in enumerate(kept)}
@@ -115,7 +128,7 @@ def tree_draft(o, n_cached: int, pend_id: int, pend_hidden, rho, Kc, Vc, topk: i
         scores=np.array([sc[c] for c in kept], np.float64),
         expanded=np.array([c in exp_k for c in kept], bool),
         k_rows=[exp_k.get(c) for c in kept], v_rows=[exp_v.get(c) for c in kept],
-        root_k=rk, root_v=rv, n_cached=P)
+        root_k=rk, root_v=rv, n_cached=P, margin=margin[0])
 
 
 def tree_verify(tree: DraftTree, target_logits: np.ndarray):

@@ -17,7 +17,7 @@ ERRORS = {0: "OK", -1: "ARG", -2: "SHAPE", -3: "DTYPE", -4: "STATE", -5: "CAPACI
 EXPORTS = ("hivis_init", "hivis_destroy", "hivis_prefill", "hivis_draft", "hivis_verify", "hivis_reset",
            "hivis_get_kv_len", "hivis_set_kv_len", "hivis_read_kv", "hivis_debug_tap", "hivis_step_bytes",
            "hivis_launch_count", "hivis_last_error", "hivis_profile_begin", "hivis_profile_end", "hivis_set_option",
-           "hivis_status", "hivis_verify_noalloc", "hivis_read_phase_times")
+           "hivis_status", "hivis_verify_noalloc", "hivis_read_phase_times", "hivis_draft_tree", "hivis_verify_tree")
 HIVIS_OPT_CHAIN_KERNEL = 0
 HIVIS_OPT_TC_KERNEL = 1
 HIVIS_OPT_WAIT_LIMIT_US = 2
@@ -76,6 +76,8 @@ def _load() -> C.CDLL:
     L.hivis_profile_begin.argtypes = [vp]
     L.hivis_profile_end.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int64)]
     L.hivis_verify_noalloc.argtypes = [i32, i32, i32, vp, vp, i32, vp, vp, vp, vp, vp]
+    L.hivis_draft_tree.argtypes = [vp, i32, i32, i32, i32, vp, i32, vp, vp, vp, vp, vp]
+    L.hivis_verify_tree.argtypes = [vp, i32, vp, i32, vp, vp, vp, vp, vp]
     L.hivis_read_phase_times.argtypes = [vp, vp, C.c_longlong, ip, ip, vp]
     L.hivis_last_error.argtypes = [vp]
     L.hivis_last_error.restype = C.c_char_p
@@ -146,6 +148,17 @@ def hivis_verify(ctx, B, seq_slots, k, draft_ids, target_logits, logits_dtype, o
     _check(lib.hivis_verify(ctx, int(B), _ints(seq_slots), int(k), _ptr(draft_ids), _ptr(target_logits),
                             int(logits_dtype), _ptr(out_accept), _ptr(out_next), _ptr(out_kv_len),
                             _stream(stream)), ctx)
+
+
+def hivis_draft_tree(ctx, slot, topk, depth, keep, resid, n_resid, out_tokens, out_parents, out_scores, out_count,
+                     stream=None):
+    _check(lib.hivis_draft_tree(ctx, int(slot), int(topk), int(depth), int(keep), _ptr(resid), int(n_resid),
+                                _ptr(out_tokens), _ptr(out_parents), _ptr(out_scores), _ptr(out_count), _stream(stream)), ctx)
+
+
+def hivis_verify_tree(ctx, slot, target_logits, logits_dtype, out_accept, out_path, out_next, out_kv_len=None, stream=None):
+    _check(lib.hivis_verify_tree(ctx, int(slot), _ptr(target_logits), int(logits_dtype), _ptr(out_accept), _ptr(out_path),
+                                 _ptr(out_next), _ptr(out_kv_len), _stream(stream)), ctx)
 
 
 def hivis_verify_noalloc(B, k, vocab, draft_ids, target_logits, logits_dtype, rows_before, out_accept,
@@ -274,6 +287,28 @@ class Drafter:
         kv = t.empty(B, dtype=t.int32, device=self.dev)
         hivis_verify(self.ctx, B, slots, k, draft_ids, target_logits, ldt, acc, nxt, kv)
         return acc, nxt, kv
+
+    def draft_tree(self, slot, topk, depth, keep, resid=None):
+        """-> (tokens, parents, scores, count) of the draft tree of one sequence; count is a 1-element tensor."""
+        t = self.torch
+        tokens = t.full((keep,), -1, dtype=t.int32, device=self.dev)
+        parents = t.full((keep,), -2, dtype=t.int32, device=self.dev)
+        scores = t.zeros((keep,), dtype=t.float32, device=self.dev)
+        count = t.zeros((4,), dtype=t.int32, device=self.dev)
+        hivis_draft_tree(self.ctx, slot, topk, depth, keep, resid, 0 if resid is None else int(resid.shape[0]), tokens,
+                         parents, scores, count)
+        return tokens, parents, scores, count
+
+    def verify_tree(self, slot, depth, target_logits):
+        """-> (n accepted, path [depth], next token, rows) tensors."""
+        t = self.torch
+        ldt = HIVIS_BF16 if target_logits.dtype == t.bfloat16 else HIVIS_F32
+        acc = t.zeros((4,), dtype=t.int32, device=self.dev)
+        path = t.full(((depth + 3) // 4 * 4,), -2, dtype=t.int32, device=self.dev)
+        nxt = t.zeros((4,), dtype=t.int32, device=self.dev)
+        kv = t.zeros((4,), dtype=t.int32, device=self.dev)
+        hivis_verify_tree(self.ctx, slot, target_logits, ldt, acc, path, nxt, kv)
+        return acc, path, nxt, kv
 
     def kv_len(self, slot):
         return hivis_get_kv_len(self.ctx, slot)

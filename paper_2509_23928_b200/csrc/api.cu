@@ -60,6 +60,12 @@ struct hivis_ctx {
     float2* rope_tab;
     int *slot_of, *row_of;
     long long map_cap;
+    // tree drafting
+    TreeBufs tree;
+    float* tree_logits;           // [TREE_MAX_TOPK][vocab] logits of the level's nodes
+    float* tree_g;                // [TREE_MAX_TOPK][d] layer outputs of the previous level
+    int tree_depth[HIVIS_MAX_BATCH];    // depth of the tree drafted last on the slot and not verified yet, else 0
+    int tree_count[HIVIS_MAX_BATCH];    // its number of kept nodes
     // host mirrors
     int kv_upper[HIVIS_MAX_BATCH];      // upper bound of the slot's row count
     bool kv_exact[HIVIS_MAX_BATCH];
@@ -305,6 +311,20 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
          dalloc(c, &c->error_flag, 2) && dalloc(c, &c->slot_of, c->map_cap) &&
          dalloc(c, &c->row_of, c->map_cap) && dalloc(c, &c->xe_h, R * d) &&
          dalloc(c, &c->rope_tab, 2 * 16 * (cfg->head_dim / 2));
+    {
+        TreeBufs& T = c->tree;
+        ok = ok && dalloc(c, &T.P, 1) && dalloc(c, &T.fr_cand, TREE_MAX_TOPK) && dalloc(c, &T.fr_tok, TREE_MAX_TOPK) &&
+             dalloc(c, &T.fr_pslot, TREE_MAX_TOPK) && dalloc(c, &T.fr_store, TREE_MAX_TOPK) &&
+             dalloc(c, &T.fr_anc, TREE_MAX_TOPK * TREE_MAX_DEPTH) && dalloc(c, &T.fr_score, TREE_MAX_TOPK) &&
+             dalloc(c, &T.top_tok, TREE_MAX_TOPK * TREE_MAX_TOPK) && dalloc(c, &T.top_lp, TREE_MAX_TOPK * TREE_MAX_TOPK) &&
+             dalloc(c, &T.cand_n, 1) && dalloc(c, &T.cand_tok, TREE_MAX_CAND) && dalloc(c, &T.cand_par, TREE_MAX_CAND) &&
+             dalloc(c, &T.cand_depth, TREE_MAX_CAND) && dalloc(c, &T.cand_store, TREE_MAX_CAND) &&
+             dalloc(c, &T.cand_keep, TREE_MAX_CAND) && dalloc(c, &T.cand_pos, TREE_MAX_CAND) &&
+             dalloc(c, &T.cand_score, TREE_MAX_CAND) && dalloc(c, &T.kept_n, 1) && dalloc(c, &T.kept_tok, HIVIS_TREE_MAX_KEEP) &&
+             dalloc(c, &T.kept_par, HIVIS_TREE_MAX_KEEP) && dalloc(c, &T.kept_store, HIVIS_TREE_MAX_KEEP) &&
+             dalloc(c, &T.row_keys, HIVIS_TREE_MAX_KEEP + 1) && dalloc(c, &c->tree_logits, (long long)TREE_MAX_TOPK * V) &&
+             dalloc(c, &c->tree_g, (long long)TREE_MAX_TOPK * d);
+    }
     if (!ok) {
         free_all(c);
         delete c;
@@ -391,6 +411,8 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
         c->pending[s] = false;
         c->have_pair[s] = false;
         c->last_k[s] = 0;
+        c->tree_depth[s] = 0;
+        c->tree_count[s] = 0;
     }
     *out = c;
     return HIVIS_OK;
@@ -487,6 +509,65 @@ static int run_qkv(hivis_ctx* c, bool mma, int b0, int nb, int row0, int N, floa
         a.xin = c->u + (long long)b0 * d;
         a.gamma = c->norm1;
         CKP(c, CLS_QKV, st, launch_gemv_alu(c->dtype, PRO_NORM, EPI_QKV, a, st));
+    }
+    return HIVIS_OK;
+}
+
+// Rows [b0, b0+nb) after the attention: O projection + residual, RMSNorm + gate/up + SiLU * up, down projection +
+// residual (-> feat, the layer output), LM head + argmax keys (logits written too when asked for).
+static int run_after_attention(hivis_ctx* c, bool mma, int b0, int nb, u64* keys_out, int keys_out_stride,
+                               float* logits_out, long long logits_ld, cudaStream_t st) {
+    const hivis_config& g = c->cfg;
+    const int d = g.d, F = g.ffn, V = g.vocab;
+    const int tiles1 = (d + HIVIS_MMA_TILE_ROWS - 1) / HIVIS_MMA_TILE_ROWS;
+    LinArgs a;
+    // ---- O projection + residual
+    memset(&a, 0, sizeof(a));
+    a.W = c->wo; a.N = d; a.K = c->qw; a.B = nb; a.ldb = c->rows_cap;
+    a.addend = c->u + (long long)b0 * d; a.out = c->y + (long long)b0 * d;
+    if (mma) {
+        a.xin_h = c->attn_h + (long long)b0 * c->qw;
+        a.out_h = c->xm + (long long)b0 * d; a.gamma_out = c->norm2; a.ssq_out = c->ssq2 + b0;
+        CKP(c, CLS_OPROJ, st, launch_gemm_mma(PRO_PLAIN, EPI_OPROJ, a, st));
+    } else {
+        a.xin = c->attn + (long long)b0 * c->qw;
+        CKP(c, CLS_OPROJ, st, launch_gemv_alu(c->dtype, PRO_PLAIN, EPI_OPROJ, a, st));
+    }
+    // ---- RMSNorm + gate/up + SiLU * up
+    memset(&a, 0, sizeof(a));
+    a.W = c->wgu; a.N = 2 * F; a.K = d; a.B = nb; a.ldb = c->rows_cap; a.eps = g.rms_eps;
+    if (mma) {
+        a.xin_h = c->xm + (long long)b0 * d; a.ssq_in = c->ssq2 + b0; a.ssq_tiles = tiles1;
+        a.out_h = c->act_h + (long long)b0 * F;
+        CKP(c, CLS_GATEUP, st, launch_gemm_mma(PRO_PLAIN, EPI_GATEUP, a, st));
+    } else {
+        a.xin = c->y + (long long)b0 * d; a.gamma = c->norm2; a.out = c->act + (long long)b0 * F;
+        CKP(c, CLS_GATEUP, st, launch_gemv_alu(c->dtype, PRO_NORM, EPI_GATEUP, a, st));
+    }
+    // ---- down projection + residual -> g, carried to the next step as its feature
+    memset(&a, 0, sizeof(a));
+    a.W = c->wdown; a.N = d; a.K = F; a.B = nb; a.ldb = c->rows_cap;
+    a.addend = c->y + (long long)b0 * d; a.out = c->feat + (long long)b0 * d;
+    a.out_h = c->feat_h + (long long)b0 * d;
+    if (mma) {
+        a.xin_h = c->act_h + (long long)b0 * F;
+        CKP(c, CLS_DOWN, st, launch_gemm_mma(PRO_PLAIN, EPI_DOWN, a, st));
+    } else {
+        a.xin = c->act + (long long)b0 * F;
+        CKP(c, CLS_DOWN, st, launch_gemv_alu(c->dtype, PRO_PLAIN, EPI_DOWN, a, st));
+    }
+    // ---- LM head + argmax
+    memset(&a, 0, sizeof(a));
+    a.W = c->lm_head; a.N = V; a.K = d; a.B = nb; a.ldb = c->rows_cap;
+    a.keys_out = keys_out; a.keys_out_stride = keys_out_stride;
+    a.logits_out = logits_out;
+    a.logits_ld = logits_ld;
+    if (mma) {
+        a.xin_h = c->feat_h + (long long)b0 * d;
+        CKP(c, CLS_LM, st, launch_gemm_mma(PRO_PLAIN, EPI_LM, a, st));
+    } else {
+        a.xin = c->feat + (long long)b0 * d;
+        CKP(c, CLS_LM, st, launch_gemv_alu(c->dtype, PRO_PLAIN, EPI_LM, a, st));
     }
     return HIVIS_OK;
 }
@@ -699,57 +780,9 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
         }
         for (int b0 = 0; b0 < B; b0 += bstep) {
             const int nb = B - b0 < bstep ? B - b0 : bstep;
-            LinArgs a;
-            // ---- O projection + residual
-            memset(&a, 0, sizeof(a));
-            a.W = c->wo; a.N = d; a.K = c->qw; a.B = nb; a.ldb = c->rows_cap;
-            a.addend = c->u + (long long)b0 * d; a.out = c->y + (long long)b0 * d;
-            if (mma) {
-                a.xin_h = c->attn_h + (long long)b0 * c->qw;
-                a.out_h = c->xm + (long long)b0 * d; a.gamma_out = c->norm2; a.ssq_out = c->ssq2 + b0;
-                CKP(c, CLS_OPROJ, st, launch_gemm_mma(PRO_PLAIN, EPI_OPROJ, a, st));
-            } else {
-                a.xin = c->attn + (long long)b0 * c->qw;
-                CKP(c, CLS_OPROJ, st, launch_gemv_alu(c->dtype, PRO_PLAIN, EPI_OPROJ, a, st));
-            }
-            // ---- RMSNorm + gate/up + SiLU * up
-            memset(&a, 0, sizeof(a));
-            a.W = c->wgu; a.N = 2 * F; a.K = d; a.B = nb; a.ldb = c->rows_cap; a.eps = g.rms_eps;
-            if (mma) {
-                a.xin_h = c->xm + (long long)b0 * d; a.ssq_in = c->ssq2 + b0; a.ssq_tiles = tiles1;
-                a.out_h = c->act_h + (long long)b0 * F;
-                CKP(c, CLS_GATEUP, st, launch_gemm_mma(PRO_PLAIN, EPI_GATEUP, a, st));
-            } else {
-                a.xin = c->y + (long long)b0 * d; a.gamma = c->norm2; a.out = c->act + (long long)b0 * F;
-                CKP(c, CLS_GATEUP, st, launch_gemv_alu(c->dtype, PRO_NORM, EPI_GATEUP, a, st));
-            }
-            // ---- down projection + residual -> g, carried to the next step as its feature
-            memset(&a, 0, sizeof(a));
-            a.W = c->wdown; a.N = d; a.K = F; a.B = nb; a.ldb = c->rows_cap;
-            a.addend = c->y + (long long)b0 * d; a.out = c->feat + (long long)b0 * d;
-            a.out_h = c->feat_h + (long long)b0 * d;
-            if (mma) {
-                a.xin_h = c->act_h + (long long)b0 * F;
-                CKP(c, CLS_DOWN, st, launch_gemm_mma(PRO_PLAIN, EPI_DOWN, a, st));
-            } else {
-                a.xin = c->act + (long long)b0 * F;
-                CKP(c, CLS_DOWN, st, launch_gemv_alu(c->dtype, PRO_PLAIN, EPI_DOWN, a, st));
-            }
-            // ---- LM head + argmax
-            memset(&a, 0, sizeof(a));
-            a.W = c->lm_head; a.N = V; a.K = d; a.B = nb; a.ldb = c->rows_cap;
-            a.keys_out = c->keys + (long long)b0 * c->key_stride + s; a.keys_out_stride = c->key_stride;
-            if (out_logits) {
-                a.logits_out = out_logits + ((long long)b0 * k + s) * V;
-                a.logits_ld = (long long)k * V;
-            }
-            if (mma) {
-                a.xin_h = c->feat_h + (long long)b0 * d;
-                CKP(c, CLS_LM, st, launch_gemm_mma(PRO_PLAIN, EPI_LM, a, st));
-            } else {
-                a.xin = c->feat + (long long)b0 * d;
-                CKP(c, CLS_LM, st, launch_gemv_alu(c->dtype, PRO_PLAIN, EPI_LM, a, st));
-            }
+            rc = run_after_attention(c, mma, b0, nb, c->keys + (long long)b0 * c->key_stride + s, c->key_stride,
+                                     out_logits ? out_logits + ((long long)b0 * k + s) * V : nullptr, (long long)k * V, st);
+            if (rc) return rc;
         }
     }
     CKP(c, CLS_OTHER, st, launch_draft_finish(B, k, c->keys, c->key_stride, out_ids, st));
@@ -793,6 +826,86 @@ int hivis_verify(hivis_ctx* c, int B, const int* seq_slots_host, int k, const in
     return HIVIS_OK;
 }
 
+int hivis_draft_tree(hivis_ctx* c, int slot, int topk, int depth, int keep, const void* resid, int n_resid,
+                     int32_t* out_tokens, int32_t* out_parents, float* out_scores, int32_t* out_count, void* stream) {
+    if (!c) return HIVIS_ERR_ARG;
+    if (slot < 0 || slot >= c->cfg.max_batch) return fail(c, HIVIS_ERR_ARG, "slot %d out of range", slot);
+    if (!out_tokens || !out_parents || !out_scores || !out_count) return fail(c, HIVIS_ERR_ARG, "null output pointer");
+    if (misaligned(out_tokens) || misaligned(out_parents) || misaligned(out_scores) || misaligned(out_count) ||
+        (resid && misaligned(resid)))
+        return fail(c, HIVIS_ERR_ARG, "device pointer not 16-byte aligned");
+    if (topk < 1 || topk > HIVIS_TREE_MAX_TOPK || topk > c->cfg.vocab)
+        return fail(c, HIVIS_ERR_CAPACITY, "topk=%d outside [1,%d]", topk, HIVIS_TREE_MAX_TOPK);
+    if (depth < 1 || depth > c->cfg.max_k) return fail(c, HIVIS_ERR_CAPACITY, "depth=%d outside [1,%d]", depth, c->cfg.max_k);
+    if (keep < 1 || keep > HIVIS_TREE_MAX_KEEP) return fail(c, HIVIS_ERR_CAPACITY, "keep=%d outside [1,%d]", keep, HIVIS_TREE_MAX_KEEP);
+    if (resid && (n_resid < 1 || n_resid > HIVIS_MAX_K)) return fail(c, HIVIS_ERR_ARG, "n_resid=%d outside [1,%d]", n_resid, HIVIS_MAX_K);
+    if (!c->pending[slot]) return fail(c, HIVIS_ERR_STATE, "slot %d has no pending pair", slot);
+    const int tree_rows = 1 + (depth - 1) * topk;
+    if (c->kv_upper[slot] + tree_rows > c->cfg.max_len)
+        return fail(c, HIVIS_ERR_CAPACITY, "slot %d: %d rows + %d tree rows > max_len %d", slot, c->kv_upper[slot], tree_rows,
+                    c->cfg.max_len);
+    cudaStream_t st = (cudaStream_t)stream;
+    const hivis_config& g = c->cfg;
+    const int d = g.d, V = g.vocab;
+    int rc;
+    if (resid) {
+        rc = prepare_rho(c, resid, n_resid, st);
+        if (rc) return rc;
+    }
+    const TreeBufs& T = c->tree;
+    CKL(c, launch_tree_begin(slot, d, c->kv_len, c->pend_feat, c->pend_id, c->feat, c->feat_h, c->cur_id, c->d_slots, T, st));
+    for (int level = 0; level < depth; ++level) {
+        const int nb = level == 0 ? 1 : topk;
+        const bool mma = use_mma(c, nb, false);
+        if (level > 0) CKL(c, launch_tree_gather(nb, d, c->tree_g, T, c->feat, c->feat_h, c->cur_id, st));
+        const int row = level < n_resid - 1 ? level : n_resid - 1;
+        const float* rho = resid ? c->rho + (long long)row * d : nullptr;
+        rc = run_fuse(c, mma, 0, nb, c->feat, c->feat_h, c->cur_id, 1, nullptr, rho, st);
+        if (rc) return rc;
+        rc = run_qkv(c, mma, 0, nb, 0, c->qkvw, c->qkv, st);
+        if (rc) return rc;
+        CK(c, launch_tree_attention(c->dtype, nb, c->qkv, c->qkvw, g.n_q_heads, g.n_kv_heads, g.head_dim, g.max_len, slot,
+                                    level, T, c->inv_freq, c->Kc, c->Vc, c->attn, c->attn_h, st));
+        c->launches += 2;
+        rc = run_after_attention(c, mma, 0, nb, c->keys, c->key_stride, c->tree_logits, V, st);
+        if (rc) return rc;
+        CKL(c, launch_tree_topk(nb, c->tree_logits, V, topk, T, st));
+        CK(c, cudaMemcpyAsync(c->tree_g, c->feat, (size_t)nb * d * sizeof(float), cudaMemcpyDeviceToDevice, st));
+        CKL(c, launch_tree_select(level, depth, nb, topk, T, st));
+    }
+    CKL(c, launch_tree_finalize(keep, T, out_tokens, out_parents, out_scores, out_count, st));
+    const int total = topk + (depth - 1) * topk * topk;
+    c->pending[slot] = false;
+    c->last_k[slot] = 0;
+    c->tree_depth[slot] = depth;
+    c->tree_count[slot] = keep < total ? keep : total;
+    c->tap_B = 0;
+    return HIVIS_OK;
+}
+
+int hivis_verify_tree(hivis_ctx* c, int slot, const void* target_logits, int logits_dtype, int32_t* out_accept,
+                      int32_t* out_path, int32_t* out_next, int32_t* out_kv_len, void* stream) {
+    if (!c) return HIVIS_ERR_ARG;
+    if (slot < 0 || slot >= c->cfg.max_batch) return fail(c, HIVIS_ERR_ARG, "slot %d out of range", slot);
+    if (!target_logits || !out_accept || !out_path || !out_next) return fail(c, HIVIS_ERR_ARG, "null argument");
+    if (misaligned(target_logits) || misaligned(out_accept) || misaligned(out_path) || misaligned(out_next) ||
+        (out_kv_len && misaligned(out_kv_len)))
+        return fail(c, HIVIS_ERR_ARG, "device pointer not 16-byte aligned");
+    if (logits_dtype != HIVIS_F32 && logits_dtype != HIVIS_BF16) return fail(c, HIVIS_ERR_DTYPE, "unknown logits dtype");
+    if (c->tree_depth[slot] == 0) return fail(c, HIVIS_ERR_STATE, "slot %d: no draft tree waits for verification", slot);
+    const hivis_config& g = c->cfg;
+    CK(c, launch_tree_verify(c->dtype, logits_dtype, slot, c->tree_depth[slot], c->tree_count[slot] + 1, g.vocab, g.n_kv_heads,
+                             g.head_dim, g.max_len, c->tree, target_logits, c->Kc, c->Vc, c->kv_len, out_accept, out_path,
+                             out_next, out_kv_len, (cudaStream_t)stream));
+    c->launches += 2;
+    c->kv_upper[slot] += c->tree_depth[slot];        // at most: the root's row and depth - 1 accepted rows
+    if (c->kv_upper[slot] > g.max_len) c->kv_upper[slot] = g.max_len;
+    c->kv_exact[slot] = false;
+    c->tree_depth[slot] = 0;
+    c->tree_count[slot] = 0;
+    return HIVIS_OK;
+}
+
 int hivis_reset(hivis_ctx* c, int slot, void* stream) {
     if (!c) return HIVIS_ERR_ARG;
     if (slot < 0 || slot >= c->cfg.max_batch) return fail(c, HIVIS_ERR_ARG, "slot %d out of range", slot);
@@ -802,6 +915,7 @@ int hivis_reset(hivis_ctx* c, int slot, void* stream) {
     c->pending[slot] = false;
     c->have_pair[slot] = false;
     c->last_k[slot] = 0;
+    c->tree_depth[slot] = 0;
     return HIVIS_OK;
 }
 
@@ -828,6 +942,7 @@ int hivis_set_kv_len(hivis_ctx* c, int slot, int n_rows, int restore_pending, vo
     c->kv_exact[slot] = true;
     if (restore_pending) c->pending[slot] = true;
     c->last_k[slot] = 0;
+    c->tree_depth[slot] = 0;
     return HIVIS_OK;
 }
 

@@ -204,6 +204,42 @@ int tc_barriers_per_step();
 int tc_lo_offset(int B);
 
 // ---------------------------------------------------------------------------------------------
+// Tree drafting (kernels_tree.cu): device-side bookkeeping of one draft tree.
+// ---------------------------------------------------------------------------------------------
+#define TREE_MAX_TOPK HIVIS_TREE_MAX_TOPK
+#define TREE_MAX_DEPTH HIVIS_MAX_K
+#define TREE_MAX_CAND (TREE_MAX_TOPK + (TREE_MAX_DEPTH - 1) * TREE_MAX_TOPK * TREE_MAX_TOPK)
+struct TreeBufs {
+    int* P;                    // [1] rows the slot held when the tree was drafted (row P = the root position)
+    // the frontier of the level being run: candidate index (-1: the root), token, cumulative log-probability, row of
+    // the previous level's output that feeds it, tree row (offset from P), tree rows of its ancestors (root first)
+    int *fr_cand, *fr_tok, *fr_pslot, *fr_store, *fr_anc;      // [TOPK], ..., [TOPK][DEPTH]
+    float* fr_score;
+    int* top_tok;              // [TOPK][TOPK] the top-k tokens of every frontier node's distribution
+    float* top_lp;             //              and their log-probabilities
+    // every candidate ever proposed, in creation order
+    int *cand_n, *cand_tok, *cand_par, *cand_depth, *cand_store, *cand_keep, *cand_pos;
+    float* cand_score;
+    // the kept nodes (the draft tree handed to the caller), for the verification
+    int *kept_n, *kept_tok, *kept_par, *kept_store;
+    u64* row_keys;             // [keep + 1] argmax keys of the target's rows
+};
+cudaError_t launch_tree_begin(int slot, int d, const int* kv_len, const float* pend_feat, const int* pend_id, float* feat,
+                              bf16* feat_h, int* cur_id, int* d_slots, const TreeBufs& T, cudaStream_t st);
+cudaError_t launch_tree_gather(int nb, int d, const float* g_prev, const TreeBufs& T, float* feat, bf16* feat_h, int* cur_id,
+                               cudaStream_t st);
+cudaError_t launch_tree_attention(int dtype, int nb, const float* qkv, int ld, int Hq, int Hkv, int dh, int max_len,
+                                  int slot, int level, const TreeBufs& T, const double* inv_freq, void* Kc, void* Vc,
+                                  float* attn, bf16* attn_h, cudaStream_t st);
+cudaError_t launch_tree_topk(int nb, const float* logits, int V, int topk, const TreeBufs& T, cudaStream_t st);
+cudaError_t launch_tree_select(int level, int depth, int nb, int topk, const TreeBufs& T, cudaStream_t st);
+cudaError_t launch_tree_finalize(int keep, const TreeBufs& T, int32_t* out_tokens, int32_t* out_parents, float* out_scores,
+                                 int32_t* out_count, cudaStream_t st);
+cudaError_t launch_tree_verify(int dtype, int logits_dtype, int slot, int depth, int rows, int V, int Hkv, int dh, int max_len,
+                               const TreeBufs& T, const void* logits, void* Kc, void* Vc, int* kv_len, int32_t* out_accept,
+                               int32_t* out_path, int32_t* out_next, int32_t* out_kv_len, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------
 // Small kernels: state set-up, prefill bookkeeping, verification, layout changes, taps.
 // ---------------------------------------------------------------------------------------------
 
