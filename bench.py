@@ -227,7 +227,7 @@ class WeightCache:
 
 
 def time_workload(wl, steps: int, warmup: int, rank: int, local_rank: int, world: int, dist, weights: WeightCache,
-                  want_e2e: bool, short: bool = False):
+                  want_e2e: bool, short: bool = False, l2_keep: int = 0):
     """Prefill (untimed), then `steps` timed benchmark steps of `wl` on this rank's GPU.  Returns the pieces of the
     JSON line that belong to one workload.  short=True: device timing of the chain only (no e2e, no clock sample)."""
     import torch
@@ -239,6 +239,8 @@ def time_workload(wl, steps: int, warmup: int, rank: int, local_rank: int, world
     lens = np.diff(cu)
     B, k = wl.batch, wl.k
     dr = Drafter(wl.dims, weights.get(wl), max_batch=B, max_len=int(lens.max()) + k + 8, max_k=max(k, 8))
+    if l2_keep:
+        dr.set_l2_keep(l2_keep)
     torch.cuda.empty_cache()
     d_ids = torch.from_numpy(ids).cuda()
     d_hidden = to_dev(hidden, wl.dims.dtype)
@@ -467,6 +469,8 @@ def main():
     ap.add_argument("--workload", default=None, help="time this workload only (default: batch 1, then batch 16)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--l2-keep", type=lambda x: int(x, 0), default=0,
+                    help="mask of weight matrices the tensor-core chain kernel asks L2 to keep (HIVIS_OPT_L2_KEEP; study aid)")
     ap.add_argument("--phase-times", action="store_true",
                     help="print where a draft step of the tensor-core chain kernel goes (its own time stamps) and exit")
     args = ap.parse_args()
@@ -523,7 +527,10 @@ def main():
     if args.phase_times:
         print(json.dumps(phase_breakdown(hi.workload(args.workload or BATCH16), weights)))
         return
-    res = time_workload(wl, args.steps, args.warmup, rank, local_rank, world, dist, weights, not args.no_e2e)
+    res = time_workload(wl, args.steps, args.warmup, rank, local_rank, world, dist, weights, not args.no_e2e,
+                        l2_keep=args.l2_keep)
+    if args.l2_keep:
+        config["l2_keep_mask"] = args.l2_keep
 
     extra = {}
     if args.workload is None:

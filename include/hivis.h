@@ -231,9 +231,13 @@ int hivis_debug_tap(hivis_ctx* ctx, int which, float* out, void* stream);
  * impossible to complete, so that every wait runs into its limit: hivis_status then returns
  * HIVIS_ERR_TIMEOUT and the context is usable again.  Nothing faults or hangs.
  * HIVIS_OPT_PHASE_TIMES (default 0): 1 makes the tensor-core chain kernel write a time stamp per CTA at the
- * events listed under hivis_read_phase_times (a store per event; off, the kernel only tests a pointer).    */
+ * events listed under hivis_read_phase_times (a store per event; off, the kernel only tests a pointer).
+ * HIVIS_OPT_L2_KEEP (default 0): bit mask over the six weight matrices of a step (bit 0 fusion FC, 1 QKV, 2 O,
+ * 3 gate/up, 4 down, 5 LM head).  The tensor-core chain kernel loads the weights of the named matrices with the
+ * keep-in-L2 policy instead of streaming them through: with k chained steps in one launch a subset that fits
+ * in L2 beside the KV cache is then read from HBM once per launch rather than once per step.                */
 enum { HIVIS_OPT_CHAIN_KERNEL = 0, HIVIS_OPT_TC_KERNEL = 1, HIVIS_OPT_WAIT_LIMIT_US = 2, HIVIS_OPT_DEBUG_MISS_BARRIER = 3,
-       HIVIS_OPT_PHASE_TIMES = 4 };
+       HIVIS_OPT_PHASE_TIMES = 4, HIVIS_OPT_L2_KEEP = 5 };
 int hivis_set_option(hivis_ctx* ctx, int option, int value);
 
 /* Where the time of a draft step goes: synchronises `stream` and copies the time stamps of the LAST hivis_draft

@@ -23,6 +23,7 @@ HIVIS_OPT_TC_KERNEL = 1
 HIVIS_OPT_WAIT_LIMIT_US = 2
 HIVIS_OPT_DEBUG_MISS_BARRIER = 3
 HIVIS_OPT_PHASE_TIMES = 4
+HIVIS_OPT_L2_KEEP = 5
 HIVIS_PHASE_EVENTS = 24
 PROFILE_CLASSES = ("fuse_fc", "qkv", "attention", "o_proj", "gate_up", "down", "lm_head_argmax", "setup_finish",
                    "draft_chain")
@@ -349,6 +350,10 @@ class Drafter:
     def miss_next_barrier(self):
         """Test aid: the grid barriers of the next draft cannot complete, so its waits run out."""
         hivis_set_option(self.ctx, HIVIS_OPT_DEBUG_MISS_BARRIER, 1)
+
+    def set_l2_keep(self, mask: int):
+        """Bit p set: the tensor-core chain kernel asks L2 to keep the weights of matrix p (0 FC .. 5 LM head)."""
+        hivis_set_option(self.ctx, HIVIS_OPT_L2_KEEP, int(mask))
 
     def record_phase_times(self, on: bool = True):
         hivis_set_option(self.ctx, HIVIS_OPT_PHASE_TIMES, 1 if on else 0)

@@ -50,6 +50,7 @@ struct hivis_ctx {
     bool debug_skew;              // option HIVIS_OPT_DEBUG_MISS_BARRIER: the next draft's grid barriers cannot complete
     int opt_tc;                   // option HIVIS_OPT_TC_KERNEL: 0 off, 1 for two or more sequences, 2 always
     bool opt_phase_times;         // option HIVIS_OPT_PHASE_TIMES
+    int opt_l2_keep;              // option HIVIS_OPT_L2_KEEP: phases whose weights are asked to stay in L2
     u64* phase_t;                 // [HIVIS_MAX_K][HIVIS_PHASE_EVENTS][num_sms]
     int phase_k;                  // draft steps of the last recorded launch (0: none)
     TcMaps tc_maps;
@@ -266,6 +267,7 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
     c->tc_ok = false;
     c->tc_partial = nullptr;
     c->opt_phase_times = false;
+    c->opt_l2_keep = 0;
     c->phase_t = nullptr;
     c->phase_k = 0;
     c->tile_ctr = nullptr;
@@ -722,6 +724,7 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
         a.attn_nslot = c->nsplit_cap;
         a.bar_counter = c->bar_counter; a.bar_base = c->bar_count_host + (c->debug_skew ? (1ull << 40) : 0ull);
         a.wait_cycles = c->wait_cycles; a.error_flag = c->error_flag; a.id_flag = c->id_flag;
+        a.l2_keep = c->opt_l2_keep;
         a.phase_t = nullptr;
         if (c->opt_phase_times) {
             CK(c, cudaMemsetAsync(c->phase_t, 0, (size_t)k * HIVIS_PHASE_EVENTS * c->num_sms * sizeof(u64), st));
@@ -978,6 +981,11 @@ int hivis_set_option(hivis_ctx* c, int option, int value) {
     }
     if (option == HIVIS_OPT_PHASE_TIMES) {
         c->opt_phase_times = value != 0;
+        return HIVIS_OK;
+    }
+    if (option == HIVIS_OPT_L2_KEEP) {
+        if (value < 0 || value >= (1 << PH_COUNT)) return fail(c, HIVIS_ERR_ARG, "HIVIS_OPT_L2_KEEP takes a mask of %d bits", PH_COUNT);
+        c->opt_l2_keep = value;
         return HIVIS_OK;
     }
     return fail(c, HIVIS_ERR_ARG, "unknown option %d", option);

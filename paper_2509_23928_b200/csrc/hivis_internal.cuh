@@ -188,6 +188,7 @@ struct TcArgs {
     int* error_flag;
     int* id_flag;              // set non-zero when a token id outside [0, V) reached the embedding lookup
     u64* phase_t;              // nullable: [k][HIVIS_PHASE_EVENTS][grid] time stamps (HIVIS_OPT_PHASE_TIMES)
+    int l2_keep;               // bit p set: the weights of phase p are loaded with the keep-in-L2 policy
 };
 // fills `maps` for the given buffers; returns cudaSuccess or an error (driver entry point missing, bad shape)
 cudaError_t tc_build_maps(TcMaps* maps, const ChainPhase* ph, int d, int qw, int F, const bf16* feat_h,

@@ -509,8 +509,12 @@ __device__ bool tc_issue_attention(const TcParams& P, TcCtl* ctl, uint32_t smemA
 template <int DH, int GQ>
 __device__ void tc_producer_w(const TcParams& P, TcCtl* ctl, uint32_t smemA, int cta, int G, const TcAttInfo& ai) {
     const TcArgs& a = P.a;
-    const u64 pol_w = policy_evict_first();
+    const u64 pol_stream = policy_evict_first();
     const u64 pol_kv = policy_evict_last();       // the cache is read again at every step
+    // Weights of the phases named in l2_keep are asked to stay in L2: every CTA reads the same tiles again at the next
+    // draft step, and a subset of the matrices fits beside the caches.  The others stream through (evict first).
+    u64 pol_w = (a.l2_keep & 1) ? pol_kv : pol_stream;
+    int pol_phase = 0;
     AttCursor<GQ> first[TC_ATT_WARPS];
 #pragma unroll
     for (int w = 0; w < TC_ATT_WARPS; ++w) {
@@ -540,6 +544,10 @@ __device__ void tc_producer_w(const TcParams& P, TcCtl* ctl, uint32_t smemA, int
         if (round > 0 && !wait_mbar(saddr(&ctl->empty[slot]), (round - 1) & 1u, ctl, a.error_flag, 3)) break;
         const uint32_t bar = saddr(&ctl->full[slot]);
         mbar_expect_tx(bar, TC_A_BYTES + TC_B_BYTES);
+        if (c.p != pol_phase) {
+            pol_phase = c.p;
+            pol_w = ((a.l2_keep >> c.p) & 1) ? pol_kv : pol_stream;
+        }
         tma_load_2d(smemA + slot * TC_A_BYTES, &P.maps.m[TCM_W + c.p], c.kb * TC_BK, c.tile * TC_TM, bar, pol_w);
         cursor_next(c, a, cta, G);
         if (++slot == TC_STAGES) { slot = 0; ++round; }
