@@ -248,23 +248,22 @@ __device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, TcCtl* 
 // the parity of its phase, so whoever does not consume the ring strictly in order (the attention warps; the
 // MMA issuer after it stepped over attention items) first makes sure the stage is in the phase it means to
 // wait for: the producer arms item idx only after item idx - TC_STAGES has been handed back.
-// The count is a plain shared-memory word written after the arming by the same thread: operations of one
-// thread on the CTA's shared memory (the barrier's arrive included) take effect in program order, so a reader
-// that sees the count finds the barrier armed.  (A release/acquire pair here costs a fence per ring item.)
-__device__ __forceinline__ unsigned ld_volatile_cta_u32(const unsigned* p) {
+// The count is written after the arming by the same thread with release semantics and read with acquire
+// semantics (CTA scope), so a reader that sees the count finds the barrier armed.
+__device__ __forceinline__ unsigned ld_acquire_cta_u32(const unsigned* p) {
     unsigned v;
-    asm volatile("ld.volatile.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(saddr(p)) : "memory");
+    asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(saddr(p)) : "memory");
     return v;
 }
-__device__ __forceinline__ void st_volatile_cta_u32(unsigned* p, unsigned v) {
-    asm volatile("st.volatile.shared::cta.u32 [%0], %1;" ::"r"(saddr(p)), "r"(v) : "memory");
+__device__ __forceinline__ void st_release_cta_u32(unsigned* p, unsigned v) {
+    asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(saddr(p)), "r"(v) : "memory");
 }
 __device__ __forceinline__ bool wait_issued(TcCtl* ctl, unsigned idx, int* error_flag, int code) {
     if (poisoned(ctl)) return false;
-    if ((int)(ld_volatile_cta_u32(&ctl->issued) - idx) > 0) return true;
+    if ((int)(ld_acquire_cta_u32(&ctl->issued) - idx) > 0) return true;
     const long long t0 = clock64();
     unsigned it = 0;
-    while ((int)(ld_volatile_cta_u32(&ctl->issued) - idx) <= 0) {
+    while ((int)(ld_acquire_cta_u32(&ctl->issued) - idx) <= 0) {
         if ((++it & 63u) == 0u) {
             if (poisoned(ctl)) return false;
             if (ld_relaxed_int(error_flag) != 0) { *(volatile int*)&ctl->abort_flag = 1; return false; }
@@ -497,7 +496,7 @@ __device__ bool tc_issue_attention(const TcParams& P, TcCtl* ctl, uint32_t smemA
             if constexpr (AttSel<GQ>::mma) attm_cursor_next(cur[w], a.pos0, a.slots, HG);
             else attw_cursor_next(cur[w], a.pos0, HG);
             if (++slot == TC_STAGES) { slot = 0; ++round; }
-            st_volatile_cta_u32(&ctl->issued, round * TC_STAGES + slot);
+            st_release_cta_u32(&ctl->issued, round * TC_STAGES + slot);
         }
     }
     return true;
@@ -552,7 +551,7 @@ __device__ void tc_producer_w(const TcParams& P, TcCtl* ctl, uint32_t smemA, int
         cursor_next(c, a, cta, G);
         if (++slot == TC_STAGES) { slot = 0; ++round; }
         if (publish) {
-            st_volatile_cta_u32(&ctl->issued, round * TC_STAGES + slot);
+            st_release_cta_u32(&ctl->issued, round * TC_STAGES + slot);
             --publish;
         }
     }
