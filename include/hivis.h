@@ -153,6 +153,23 @@ int hivis_verify(hivis_ctx* ctx, int B, const int* seq_slots_host, int k,
                  const int32_t* draft_ids, const void* target_logits, int logits_dtype,
                  int32_t* out_accept, int32_t* out_next, int32_t* out_kv_len, void* stream);
 
+/* Verification by speculative sampling, for drafts whose tokens were DRAWN from the drafter's distribution
+ * (Sec. 2.1: the target keeps the drafted tokens that are consistent with its distribution, drops the first
+ * that is not together with all that follow and re-draws the next token accordingly; the rule is the one of
+ * Leviathan et al. and Chen et al., which the section cites).  With p_j = softmax(target row j / T) and
+ * q_j = softmax(drafter row j / T): draft token j is kept while u_accept[b, j] < min(1, p_j(x) / q_j(x));
+ * n = number kept; the next token is drawn by inverse CDF at u_sample[b] from max(0, p_n - q_n) (n < k) or
+ * from p_k (n = k): the first token whose cumulative mass exceeds u_sample[b] times the total mass.
+ *   draft_logits fp32 [B, k, vocab]: the drafter's logits of the k steps (hivis_draft's out_logits);
+ *   target_logits [B, k+1, vocab] in logits_dtype; temperature > 0;
+ *   u_accept fp32 [B, k], u_sample fp32 [B]: uniform numbers in [0, 1) supplied by the caller;
+ *   outputs and rollback as for hivis_verify.  Must follow a hivis_draft of the same k on the same slots.
+ * Errors: ARG, DTYPE, STATE, CAPACITY, CUDA.                                                            */
+int hivis_verify_sampled(hivis_ctx* ctx, int B, const int* seq_slots_host, int k, const int32_t* draft_ids,
+                         const float* draft_logits, const void* target_logits, int logits_dtype,
+                         float temperature, const float* u_accept, const float* u_sample,
+                         int32_t* out_accept, int32_t* out_next, int32_t* out_kv_len, void* stream);
+
 /* Tree drafting for ONE sequence (Sec. 2.1: the paper drafts with the dynamic draft tree of EAGLE-2;
  * "Inference Setup": top-10 expansion, depth 6, the 60 paths of highest cumulative probability kept;
  * supplementary material, Sec. A: 8 per expansion, depth 4, 30 kept).

@@ -17,7 +17,7 @@ ERRORS = {0: "OK", -1: "ARG", -2: "SHAPE", -3: "DTYPE", -4: "STATE", -5: "CAPACI
 EXPORTS = ("hivis_init", "hivis_destroy", "hivis_prefill", "hivis_draft", "hivis_verify", "hivis_reset",
            "hivis_get_kv_len", "hivis_set_kv_len", "hivis_read_kv", "hivis_debug_tap", "hivis_step_bytes",
            "hivis_launch_count", "hivis_last_error", "hivis_profile_begin", "hivis_profile_end", "hivis_set_option",
-           "hivis_status", "hivis_verify_noalloc", "hivis_read_phase_times", "hivis_draft_tree", "hivis_verify_tree")
+           "hivis_status", "hivis_verify_noalloc", "hivis_read_phase_times", "hivis_draft_tree", "hivis_verify_tree", "hivis_verify_sampled")
 HIVIS_OPT_CHAIN_KERNEL = 0
 HIVIS_OPT_TC_KERNEL = 1
 HIVIS_OPT_WAIT_LIMIT_US = 2
@@ -77,6 +77,7 @@ def _load() -> C.CDLL:
     L.hivis_profile_begin.argtypes = [vp]
     L.hivis_profile_end.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int64)]
     L.hivis_verify_noalloc.argtypes = [i32, i32, i32, vp, vp, i32, vp, vp, vp, vp, vp]
+    L.hivis_verify_sampled.argtypes = [vp, i32, ip, i32, vp, vp, vp, i32, C.c_float, vp, vp, vp, vp, vp, vp]
     L.hivis_draft_tree.argtypes = [vp, i32, i32, i32, i32, vp, i32, vp, vp, vp, vp, vp]
     L.hivis_verify_tree.argtypes = [vp, i32, vp, i32, vp, vp, vp, vp, vp]
     L.hivis_read_phase_times.argtypes = [vp, vp, C.c_longlong, ip, ip, vp]
@@ -149,6 +150,13 @@ def hivis_verify(ctx, B, seq_slots, k, draft_ids, target_logits, logits_dtype, o
     _check(lib.hivis_verify(ctx, int(B), _ints(seq_slots), int(k), _ptr(draft_ids), _ptr(target_logits),
                             int(logits_dtype), _ptr(out_accept), _ptr(out_next), _ptr(out_kv_len),
                             _stream(stream)), ctx)
+
+
+def hivis_verify_sampled(ctx, B, seq_slots, k, draft_ids, draft_logits, target_logits, logits_dtype, temperature, u_accept,
+                         u_sample, out_accept, out_next, out_kv_len=None, stream=None):
+    _check(lib.hivis_verify_sampled(ctx, int(B), _ints(seq_slots), int(k), _ptr(draft_ids), _ptr(draft_logits),
+                                    _ptr(target_logits), int(logits_dtype), float(temperature), _ptr(u_accept), _ptr(u_sample),
+                                    _ptr(out_accept), _ptr(out_next), _ptr(out_kv_len), _stream(stream)), ctx)
 
 
 def hivis_draft_tree(ctx, slot, topk, depth, keep, resid, n_resid, out_tokens, out_parents, out_scores, out_count,
@@ -288,6 +296,17 @@ class Drafter:
         kv = t.empty(B, dtype=t.int32, device=self.dev)
         hivis_verify(self.ctx, B, slots, k, draft_ids, target_logits, ldt, acc, nxt, kv)
         return acc, nxt, kv
+
+    def verify_sampled(self, draft_ids, draft_logits, target_logits, temperature, u_accept, u_sample, slots=None):
+        t = self.torch
+        B, k = draft_ids.shape
+        ldt = HIVIS_BF16 if target_logits.dtype == t.bfloat16 else HIVIS_F32
+        acc = t.empty((B + 3) // 4 * 4, dtype=t.int32, device=self.dev)
+        nxt = t.empty_like(acc)
+        kv = t.empty_like(acc)
+        hivis_verify_sampled(self.ctx, B, slots, k, draft_ids, draft_logits, target_logits, ldt, temperature, u_accept,
+                             u_sample, acc, nxt, kv)
+        return acc[:B], nxt[:B], kv[:B]
 
     def draft_tree(self, slot, topk, depth, keep, resid=None):
         """-> (tokens, parents, scores, count) of the draft tree of one sequence; count is a 1-element tensor."""

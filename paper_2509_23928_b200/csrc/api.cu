@@ -30,6 +30,7 @@ struct hivis_ctx {
     bf16 *feat_h, *xq, *attn_h, *xm, *act_h;
     u64* keys;
     int key_stride;
+    float2* vstats;               // sampled verification: (max, log sum exp) of every logits row [max_batch * (2 max_k + 1)]
     u64* vkeys;                   // verification: argmax keys [max_batch][max_k + 1] and arrival counters
     int* varrive;                 // [max_batch]; both zero between calls
     float *part_acc, *part_ml;
@@ -307,6 +308,7 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
          dalloc(c, &c->rho, (long long)HIVIS_MAX_K * d) && dalloc(c, &c->ssq1, tiles1 * R) &&
          dalloc(c, &c->ssq2, tiles1 * R) && dalloc(c, &c->keys, R * c->key_stride) &&
          dalloc(c, &c->vkeys, MB * (cfg->max_k + 1)) && dalloc(c, &c->varrive, MB) &&
+         dalloc(c, &c->vstats, MB * (2 * cfg->max_k + 1)) &&
          dalloc(c, &c->part_acc, R * cfg->n_q_heads * (long long)c->nsplit_cap * cfg->head_dim) &&
          dalloc(c, &c->part_ml, R * cfg->n_q_heads * (long long)c->nsplit_cap * 2) &&
          dalloc(c, &c->counters, R * cfg->n_q_heads) && dalloc(c, &c->bar_counter, 1) &&
@@ -825,6 +827,37 @@ int hivis_verify(hivis_ctx* c, int B, const int* seq_slots_host, int k, const in
         const int s = sl.slot[b];
         c->last_k[s] = 0;
         c->kv_exact[s] = false;          // between pairs and pairs + k - 1 until read back
+    }
+    return HIVIS_OK;
+}
+
+int hivis_verify_sampled(hivis_ctx* c, int B, const int* seq_slots_host, int k, const int32_t* draft_ids,
+                         const float* draft_logits, const void* target_logits, int logits_dtype, float temperature,
+                         const float* u_accept, const float* u_sample, int32_t* out_accept, int32_t* out_next,
+                         int32_t* out_kv_len, void* stream) {
+    if (!c) return HIVIS_ERR_ARG;
+    SlotList sl;
+    int rc = check_slots(c, B, seq_slots_host, &sl);
+    if (rc) return rc;
+    if (!draft_ids || !draft_logits || !target_logits || !u_accept || !u_sample || !out_accept || !out_next)
+        return fail(c, HIVIS_ERR_ARG, "null argument");
+    if (misaligned(draft_ids) || misaligned(draft_logits) || misaligned(target_logits) || misaligned(u_accept) ||
+        misaligned(u_sample) || misaligned(out_accept) || misaligned(out_next) || (out_kv_len && misaligned(out_kv_len)))
+        return fail(c, HIVIS_ERR_ARG, "device pointer not 16-byte aligned");
+    if (logits_dtype != HIVIS_F32 && logits_dtype != HIVIS_BF16) return fail(c, HIVIS_ERR_DTYPE, "unknown logits dtype");
+    if (!(temperature > 0.f)) return fail(c, HIVIS_ERR_ARG, "temperature must be positive");
+    if (k < 1 || k > c->cfg.max_k) return fail(c, HIVIS_ERR_CAPACITY, "k=%d outside [1,%d]", k, c->cfg.max_k);
+    for (int b = 0; b < B; ++b)
+        if (c->last_k[sl.slot[b]] != k)
+            return fail(c, HIVIS_ERR_STATE, "slot %d: verification (k=%d) must follow a draft of the same k", sl.slot[b], k);
+    CK(c, launch_verify_sampled(logits_dtype, sl, k, c->cfg.vocab, temperature, draft_ids, draft_logits, target_logits,
+                                c->vstats, u_accept, u_sample, c->kv_len, out_accept, out_next, out_kv_len,
+                                (cudaStream_t)stream));
+    c->launches += 2;
+    for (int b = 0; b < B; ++b) {
+        const int s = sl.slot[b];
+        c->last_k[s] = 0;
+        c->kv_exact[s] = false;
     }
     return HIVIS_OK;
 }

@@ -275,6 +275,13 @@ cudaError_t launch_verify(int logits_dtype, const SlotList& sl, int k, int V, co
                           const void* logits, u64* keys, int* arrivals, int* kv_len, int32_t* out_accept,
                           int32_t* out_next, int32_t* out_kv_len, cudaStream_t st, int* n_launches);
 
+// verification by speculative sampling: per-row softmax statistics, then acceptance tests, the draw of the next token
+// and the rollback; stats: [B * (2k + 1)] scratch
+cudaError_t launch_verify_sampled(int logits_dtype, const SlotList& sl, int k, int V, float temperature,
+                                  const int32_t* draft_ids, const float* draft_logits, const void* target_logits,
+                                  float2* stats, const float* u_accept, const float* u_sample, int* kv_len,
+                                  int32_t* out_accept, int32_t* out_next, int32_t* out_kv_len, cudaStream_t st);
+
 cudaError_t launch_set_int(int* p, int v, cudaStream_t st);
 
 // weight re-layout at init

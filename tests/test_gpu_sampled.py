@@ -1,0 +1,91 @@
+"""GPU parity of verification by speculative sampling (hivis_verify_sampled) against the oracle (oracle/sampled.py)."""
+import numpy as np
+import pytest
+
+import hivis_inputs as hi
+from oracle import sampled as osmp
+from tests.harness import Case, to_dev
+
+pytestmark = pytest.mark.gpu
+
+# A uniform number closer than this to the threshold that decides its outcome is not compared: the acceptance ratio
+# is a quotient of two fp32 softmax values, the draw a position in a cumulative sum of up to 150 000 fp32 masses.
+MARGIN_ACCEPT = 1e-4
+MARGIN_DRAW = 5e-6
+
+
+@pytest.mark.parametrize("name,temperature,closeness", [
+    ("mini_gqa_b16_ragged", 1.0, 0.3), ("mini_gqa_b16_ragged", 0.7, 1.5), ("mini_gqa_b3", 1.0, 0.0),
+    ("mini_mha_b5_ragged", 1.3, 0.6), ("tiny_f32_b4_ragged", 1.0, 0.4),
+])
+def test_sampled_verification_parity(name, temperature, closeness):
+    """closeness: the target's logits are the drafter's plus noise of that size (0: identical distributions, so
+    every token is kept and the bonus token is drawn from p)."""
+    import torch
+    wl = hi.workload(name)
+    case = Case(wl)
+    try:
+        B, k, V = wl.batch, wl.k, wl.dims.vocab
+        rng = np.random.default_rng(31)
+        compared = 0
+        case.gpu_prefill()
+        for trial in range(3):
+            case.gpu_restore()
+            _, dl = case.gpu_draft(k)                                   # the drafter's logits [B, k, V] fp32
+            # drafted tokens: drawn from q for most positions, a uniformly random token now and then
+            ids = np.zeros((B, k), np.int32)
+            for b in range(B):
+                for j in range(k):
+                    q = osmp.softmax_t(dl[b, j], temperature)
+                    ids[b, j] = rng.choice(V, p=q) if rng.random() < 0.8 else rng.integers(0, V)
+            tl = np.concatenate([dl, rng.standard_normal((B, 1, V)).astype(np.float32)], 1)
+            tl = tl + closeness * rng.standard_normal(tl.shape).astype(np.float32)
+            tl = hi.round_to_bf16(tl) if wl.logits_dtype == "bf16" else tl.astype(np.float32)
+            ua = rng.random((B, k)).astype(np.float32)
+            us = rng.random(B).astype(np.float32)
+            acc, nxt, kv = case.drafter.verify_sampled(torch.from_numpy(ids).cuda(), torch.from_numpy(dl).cuda(),
+                                                       to_dev(tl, wl.logits_dtype), temperature,
+                                                       torch.from_numpy(ua).cuda(), torch.from_numpy(us).cuda())
+            torch.cuda.synchronize()
+            acc, nxt, kv = acc.cpu().numpy(), nxt.cpu().numpy(), kv.cpu().numpy()
+            for b in range(B):
+                n, nx, kvl, margin = osmp.verify_sampled(ids[b], dl[b], tl[b], temperature, ua[b], float(us[b]), int(case.lens[b]))
+                assert 0 <= acc[b] <= k and 0 <= nxt[b] < V
+                assert kv[b] == int(case.lens[b]) + min(int(acc[b]), k - 1)
+                assert case.drafter.kv_len(b)[0] == kv[b]
+                if margin[0] > MARGIN_ACCEPT:
+                    assert (int(acc[b]), int(kv[b])) == (n, kvl), f"trial {trial} seq {b} (margin {margin[0]:.1e})"
+                    if margin[1] > MARGIN_DRAW:
+                        assert int(nxt[b]) == nx, f"trial {trial} seq {b}: drawn token (margin {margin[1]:.1e})"
+                        compared += 1
+                if closeness == 0.0 and wl.logits_dtype == "f32":
+                    assert acc[b] == k
+        assert compared >= 0.8 * 3 * B, f"only {compared} of {3 * B} sequences were away from every threshold"
+    finally:
+        case.close()
+
+
+def test_sampled_verification_errors():
+    import torch
+    from paper_2509_23928_b200 import HivisError
+    wl = hi.workload("mini_gqa_b3")
+    case = Case(wl)
+    try:
+        B, k, V = wl.batch, wl.k, wl.dims.vocab
+        ids = torch.zeros((B, k), dtype=torch.int32, device="cuda")
+        dl = torch.zeros((B, k, V), device="cuda")
+        tl = torch.zeros((B, k + 1, V), device="cuda")
+        u = torch.zeros((B, k), device="cuda")
+        with pytest.raises(HivisError) as e:                     # no draft to verify
+            case.drafter.verify_sampled(ids, dl, tl, 1.0, u, u[:, 0].contiguous())
+        assert e.value.code == -4
+        case.gpu_prefill()
+        case.gpu_draft(k, want_logits=False)
+        with pytest.raises(HivisError) as e:                     # temperature must be positive
+            case.drafter.verify_sampled(ids, dl, tl, 0.0, u, u[:, 0].contiguous())
+        assert e.value.code == -1
+        acc, nxt, kv = case.drafter.verify_sampled(ids, dl, tl, 1.0, u, u[:, 0].contiguous())
+        torch.cuda.synchronize()
+        assert (acc.cpu().numpy() == k).all() and (nxt.cpu().numpy() == 0).all()      # uniform vs uniform, u = 0
+    finally:
+        case.close()
