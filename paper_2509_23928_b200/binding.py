@@ -24,6 +24,7 @@ HIVIS_OPT_WAIT_LIMIT_US = 2
 HIVIS_OPT_DEBUG_MISS_BARRIER = 3
 HIVIS_OPT_PHASE_TIMES = 4
 HIVIS_OPT_L2_KEEP = 5
+HIVIS_OPT_TC_PREFILL = 6
 HIVIS_PHASE_EVENTS = 24
 PROFILE_CLASSES = ("fuse_fc", "qkv", "attention", "o_proj", "gate_up", "down", "lm_head_argmax", "setup_finish",
                    "draft_chain")
@@ -369,6 +370,10 @@ class Drafter:
     def miss_next_barrier(self):
         """Test aid: the grid barriers of the next draft cannot complete, so its waits run out."""
         hivis_set_option(self.ctx, HIVIS_OPT_DEBUG_MISS_BARRIER, 1)
+
+    def set_tc_prefill(self, on: bool):
+        """False: hivis_prefill always uses the 16-pairs-per-pass kernels."""
+        hivis_set_option(self.ctx, HIVIS_OPT_TC_PREFILL, 1 if on else 0)
 
     def set_l2_keep(self, mask: int):
         """Bit p set: the tensor-core chain kernel asks L2 to keep the weights of matrix p (0 FC .. 5 LM head)."""

@@ -52,6 +52,10 @@ struct hivis_ctx {
     int opt_tc;                   // option HIVIS_OPT_TC_KERNEL: 0 off, 1 for two or more sequences, 2 always
     bool opt_phase_times;         // option HIVIS_OPT_PHASE_TIMES
     int opt_l2_keep;              // option HIVIS_OPT_L2_KEEP: phases whose weights are asked to stay in L2
+    bool opt_tc_prefill;          // option HIVIS_OPT_TC_PREFILL
+    bool pf_ok;                   // the tensor-core prefill can run (bf16, shapes, buffers)
+    bf16 *pf_xe, *pf_xq;          // [map_cap][d] pair-major operands of the tensor-core prefill
+    float* pf_ssq;                // [ceil(d / 128)][map_cap]
     u64* phase_t;                 // [HIVIS_MAX_K][HIVIS_PHASE_EVENTS][num_sms]
     int phase_k;                  // draft steps of the last recorded launch (0: none)
     TcMaps tc_maps;
@@ -269,6 +273,10 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
     c->tc_partial = nullptr;
     c->opt_phase_times = false;
     c->opt_l2_keep = 0;
+    c->opt_tc_prefill = true;
+    c->pf_ok = false;
+    c->pf_xe = c->pf_xq = nullptr;
+    c->pf_ssq = nullptr;
     c->phase_t = nullptr;
     c->phase_k = 0;
     c->tile_ctr = nullptr;
@@ -408,6 +416,10 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
                                 cfg->head_dim) == cudaSuccess;
         if (!ok2) cudaGetLastError();
         c->tc_ok = ok2;
+    }
+    if (c->dtype == HIVIS_BF16 && prefill_tc_supported(cfg->d, c->kvw)) {
+        c->pf_ok = dalloc(c, &c->pf_xe, (size_t)c->map_cap * d) && dalloc(c, &c->pf_xq, (size_t)c->map_cap * d) &&
+                   dalloc(c, &c->pf_ssq, (size_t)((d + 127) / 128) * c->map_cap);
     }
     for (int s = 0; s < HIVIS_MAX_BATCH; ++s) {
         c->kv_upper[s] = 0;
@@ -623,6 +635,24 @@ int hivis_prefill(hivis_ctx* c, int B, const int* seq_slots_host, const int32_t*
     }
     CKL(c, launch_prefill_setup(c->dtype, sl, cu, start, d, ids, hidden, c->kv_len, c->pend_feat, c->pend_id,
                                 c->slot_of, c->row_of, st));
+    if (c->pf_ok && c->opt_tc_prefill && total >= 128) {
+        // many pairs: the two GEMMs of the prefix build on the tensor cores, all pairs in one pass
+        PrefillTcArgs a;
+        memset(&a, 0, sizeof(a));
+        a.n_pairs = (int)total; a.pair_cap = (int)c->map_cap;
+        a.d = d; a.kvw = c->kvw; a.Hkv = c->cfg.n_kv_heads; a.dh = c->cfg.head_dim; a.max_len = c->cfg.max_len;
+        a.vocab = c->cfg.vocab; a.eps = c->cfg.rms_eps;
+        a.ids = ids; a.hidden = (const bf16*)hidden; a.embed = (const bf16*)c->embed; a.fc = (const bf16*)c->fc;
+        a.wkv = (const bf16*)c->wqkv + (long long)c->qw * d;
+        a.bkv = c->bqkv ? (const bf16*)c->bqkv + c->qw : nullptr;
+        a.norm1 = (const bf16*)c->norm1; a.rho0 = rho0;
+        a.xe = c->pf_xe; a.xq = c->pf_xq; a.ssq = c->pf_ssq;
+        a.slot_of = c->slot_of; a.row_of = c->row_of; a.inv_freq = c->inv_freq;
+        a.Kc = (bf16*)c->Kc; a.Vc = (bf16*)c->Vc;
+        a.wait_cycles = c->wait_cycles; a.error_flag = c->error_flag; a.id_flag = c->id_flag;
+        CK(c, launch_prefill_tc(a, st));
+        c->launches += 3;
+    } else {
     const bool mma = use_mma(c, 16, true);
     for (long long j0 = 0; j0 < total; j0 += 16) {
         const int P = (int)(total - j0 < 16 ? total - j0 : 16);
@@ -634,6 +664,7 @@ int hivis_prefill(hivis_ctx* c, int B, const int* seq_slots_host, const int32_t*
         if (rc) return rc;
         CKL(c, launch_kv_append(c->dtype, c->qkv, P, c->slot_of + j0, c->row_of + j0, c->inv_freq,
                                 c->cfg.n_kv_heads, c->cfg.head_dim, c->cfg.max_len, c->Kc, c->Vc, st));
+    }
     }
     for (int b = 0; b < B; ++b) {
         const int s = sl.slot[b];
@@ -1014,6 +1045,10 @@ int hivis_set_option(hivis_ctx* c, int option, int value) {
     }
     if (option == HIVIS_OPT_PHASE_TIMES) {
         c->opt_phase_times = value != 0;
+        return HIVIS_OK;
+    }
+    if (option == HIVIS_OPT_TC_PREFILL) {
+        c->opt_tc_prefill = value != 0;
         return HIVIS_OK;
     }
     if (option == HIVIS_OPT_L2_KEEP) {

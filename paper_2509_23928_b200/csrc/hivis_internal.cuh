@@ -205,6 +205,28 @@ int tc_barriers_per_step();
 int tc_lo_offset(int B);
 
 // ---------------------------------------------------------------------------------------------
+// Prefix build on the tensor cores (kernels_prefill_tc.cu): two tcgen05 GEMMs over all packed pairs.
+// ---------------------------------------------------------------------------------------------
+struct PrefillTcArgs {
+    int n_pairs, pair_cap;     // packed pairs of the call; capacity of the pair-major buffers
+    int d, kvw, Hkv, dh, max_len, vocab;
+    float eps;
+    const int32_t* ids;        // [n_pairs]
+    const bf16* hidden;        // [n_pairs][d] the caller's hidden states
+    const bf16 *embed, *fc, *wkv, *bkv, *norm1;      // wkv: rows [K ; V] of the stacked QKV matrix, bkv nullable
+    const float* rho0;         // [d] nullable
+    bf16 *xe, *xq;             // [pair_cap][d] gathered embedding rows; gamma_1 * u
+    float* ssq;                // [ceil(d / 128)][pair_cap]
+    const int *slot_of, *row_of;
+    const double* inv_freq;
+    bf16 *Kc, *Vc;
+    long long wait_cycles;
+    int *error_flag, *id_flag;
+};
+bool prefill_tc_supported(int d, int kvw);
+cudaError_t launch_prefill_tc(const PrefillTcArgs& a, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------
 // Tree drafting (kernels_tree.cu): device-side bookkeeping of one draft tree.
 // ---------------------------------------------------------------------------------------------
 #define TREE_MAX_TOPK HIVIS_TREE_MAX_TOPK

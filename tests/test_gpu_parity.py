@@ -208,6 +208,45 @@ def test_nan_hidden_state_gives_token_zero_on_both_sides(name, tc):
         case.close()
 
 
+@pytest.mark.parametrize("name", ["mini_gqa_b16_ragged", "mini_mha_b5_ragged", "gqa4_b16_ragged", "wide_gqa_b16_ragged"])
+def test_tensor_core_prefill_against_oracle_and_per_pass_prefill(name):
+    """The prefix build as two tcgen05 GEMMs over all pairs (calls of 128 pairs or more) and the 16-pairs-per-pass
+    kernels: the cached K/V rows of both against the oracle's, and the draft that follows."""
+    import torch
+    wl = hi.workload(name)
+    case = Case(wl)
+    try:
+        assert int(case.cu[-1]) >= 128
+        ref = case.oracle_run()
+        rows = {}
+        for tc_prefill in (True, False):
+            case.drafter.set_tc_prefill(tc_prefill)
+            case.drafter.prefill(case.d_ids, case.d_hidden, [int(x) for x in case.cu], start_pos=[0] * wl.batch,
+                                 resid0=case.d_resid[0])
+            case.drafter.status()
+            for b in range(wl.batch):
+                n = int(case.lens[b]) - 1
+                if n == 0:
+                    continue
+                k_g, v_g = case.drafter.read_kv(b, 0, n)
+                torch.cuda.synchronize()
+                for got, want, nm in ((k_g, ref[b]["K"][:n], "K"), (v_g, ref[b]["V"][:n], "V")):
+                    e = np.abs(got.cpu().numpy() - want).max() / np.abs(want).max()
+                    assert e <= 1e-2, f"tc_prefill={tc_prefill} {nm} cache of seq {b}: rel err {e}"
+                rows[(tc_prefill, b)] = (k_g.cpu().numpy(), v_g.cpu().numpy())
+        for b in range(wl.batch):
+            if (True, b) in rows:
+                for x, y in zip(rows[(True, b)], rows[(False, b)]):
+                    assert np.abs(x - y).max() / np.abs(y).max() <= 1e-2
+        case.drafter.set_tc_prefill(True)
+        for b in range(wl.batch):
+            case.drafter.reset(b)
+        res = check_draft_parity(case)                 # prefill (tensor-core path) + draft against the oracle
+        check_kv_parity(case, res["ref"])
+    finally:
+        case.close()
+
+
 def test_more_sequences_than_the_chain_kernels_take():
     """20 sequences: beyond the 16 of the tensor-core chain kernel, so the per-phase kernels run in two passes."""
     wl = hi.scaled(hi.workload("mini_gqa_b16_ragged"), batch=20, k=3, seed=2103)
