@@ -457,6 +457,59 @@ def phase_breakdown(wl, weights: WeightCache, reps: int = 20):
     return out
 
 
+def prefill_ablation(reps: int = 5):
+    """The visual-token-hiding ablation on the prefix build: time of hivis_prefill for the LLaVA-shaped drafter at batch 16
+    with 128 text positions and 0 (text-only), 576 or 2048 leading positions standing in for visual tokens, on the
+    tensor-core path and on the 16-pairs-per-pass path.  CUDA events around the call, median of `reps`."""
+    import torch
+    from hivis_inputs.device import to_dev
+    from paper_2509_23928_b200 import Drafter
+    base = hi.workload(BATCH16)
+    weights = WeightCache()
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    tf_peak = float(peaks.get("bf16_tflops", 1590.0))
+    out = {"workload": "LLaVA-shaped drafter, batch 16, 128 text positions + leading positions", "unit": "ms per hivis_prefill call",
+           "tensor_peak_tflops": tf_peak, "tensor_peak_kind": "measured" if "bf16_tflops" in peaks else "fallback", "rows": []}
+    for lead in (0, 576, 2048):
+        wl = hi.scaled(base, leading_positions=lead, name=f"llava_b16_lead{lead}")
+        ids, hidden, cu = hi.make_prompt(wl)
+        resid = hi.make_residuals(wl)
+        lens = np.diff(cu)
+        B, k, D = wl.batch, wl.k, wl.dims
+        dr = Drafter(D, weights.get(wl), max_batch=B, max_len=int(lens.max()) + k + 8, max_k=8)
+        d_ids = torch.from_numpy(ids).cuda()
+        d_hidden = to_dev(hidden, D.dtype)
+        d_resid = to_dev(resid, D.dtype)
+        pairs = int(cu[-1])
+        flops = 2.0 * pairs * (2 * D.d * D.d + D.d * 2 * D.kv_dim)
+        row = {"leading_positions": lead, "pairs": pairs}
+        for label, on in (("tensor_core", True), ("per_pass", False)):
+            dr.set_tc_prefill(on)
+            ts = []
+            for it in range(reps + 2):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                dr.prefill(d_ids, d_hidden, [int(x) for x in cu], start_pos=[0] * B, resid0=d_resid[0])
+                e1.record()
+                torch.cuda.synchronize()
+                if it >= 2:
+                    ts.append(e0.elapsed_time(e1))
+            ms = float(np.median(ts))
+            row[label] = {"ms": round(ms, 3), "pairs_per_s": round(pairs / (ms * 1e-3)), "tflops": round(flops / (ms * 1e-3) / 1e12, 1),
+                          "frac_of_tensor_peak": round(flops / (ms * 1e-3) / 1e12 / tf_peak, 4)}
+        dr.status()
+        dr.close()
+        out["rows"].append(row)
+    t0 = out["rows"][0]["tensor_core"]["ms"]
+    for r in out["rows"]:
+        r["tensor_core_over_text_only"] = round(r["tensor_core"]["ms"] / t0, 2)
+    return out
+
+
 def stub_replica(rank: int) -> dict:
     """Stands in for the device work when HIVIS_BENCH_STUB=1 (CPU test of the launch path only): fixed fake
     times, rank 1 slower.  The line it leads to is marked as a stub and carries no measurement."""
@@ -474,6 +527,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--l2-keep", type=lambda x: int(x, 0), default=0,
                     help="mask of weight matrices the tensor-core chain kernel asks L2 to keep (HIVIS_OPT_L2_KEEP; study aid)")
+    ap.add_argument("--prefill-ablation", action="store_true",
+                    help="time the prefix build with 0 / 576 / 2048 leading (visual stand-in) positions and exit")
     ap.add_argument("--phase-times", action="store_true",
                     help="print where a draft step of the tensor-core chain kernel goes (its own time stamps) and exit")
     args = ap.parse_args()
@@ -527,6 +582,9 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     wl = replica_workload(wl, rank, world)                 # independent replicas, same shapes
     weights = WeightCache()
+    if args.prefill_ablation:
+        print(json.dumps(prefill_ablation()))
+        return
     if args.phase_times:
         print(json.dumps(phase_breakdown(hi.workload(args.workload or BATCH16), weights)))
         return

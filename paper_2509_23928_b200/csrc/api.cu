@@ -56,6 +56,7 @@ struct hivis_ctx {
     bool pf_ok;                   // the tensor-core prefill can run (bf16, shapes, buffers)
     bf16 *pf_xe, *pf_xq;          // [map_cap][d] pair-major operands of the tensor-core prefill
     float* pf_ssq;                // [ceil(d / 128)][map_cap]
+    float2* pf_rope;              // [map_cap][head_dim / 2]
     u64* phase_t;                 // [HIVIS_MAX_K][HIVIS_PHASE_EVENTS][num_sms]
     int phase_k;                  // draft steps of the last recorded launch (0: none)
     TcMaps tc_maps;
@@ -419,7 +420,8 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
     }
     if (c->dtype == HIVIS_BF16 && prefill_tc_supported(cfg->d, c->kvw)) {
         c->pf_ok = dalloc(c, &c->pf_xe, (size_t)c->map_cap * d) && dalloc(c, &c->pf_xq, (size_t)c->map_cap * d) &&
-                   dalloc(c, &c->pf_ssq, (size_t)((d + 127) / 128) * c->map_cap);
+                   dalloc(c, &c->pf_ssq, (size_t)((d + 127) / 128) * c->map_cap) &&
+                   dalloc(c, &c->pf_rope, (size_t)c->map_cap * (cfg->head_dim / 2));
     }
     for (int s = 0; s < HIVIS_MAX_BATCH; ++s) {
         c->kv_upper[s] = 0;
@@ -646,12 +648,12 @@ int hivis_prefill(hivis_ctx* c, int B, const int* seq_slots_host, const int32_t*
         a.wkv = (const bf16*)c->wqkv + (long long)c->qw * d;
         a.bkv = c->bqkv ? (const bf16*)c->bqkv + c->qw : nullptr;
         a.norm1 = (const bf16*)c->norm1; a.rho0 = rho0;
-        a.xe = c->pf_xe; a.xq = c->pf_xq; a.ssq = c->pf_ssq;
+        a.xe = c->pf_xe; a.xq = c->pf_xq; a.ssq = c->pf_ssq; a.rope = c->pf_rope;
         a.slot_of = c->slot_of; a.row_of = c->row_of; a.inv_freq = c->inv_freq;
         a.Kc = (bf16*)c->Kc; a.Vc = (bf16*)c->Vc;
         a.wait_cycles = c->wait_cycles; a.error_flag = c->error_flag; a.id_flag = c->id_flag;
         CK(c, launch_prefill_tc(a, st));
-        c->launches += 3;
+        c->launches += 4;
     } else {
     const bool mma = use_mma(c, 16, true);
     for (long long j0 = 0; j0 < total; j0 += 16) {

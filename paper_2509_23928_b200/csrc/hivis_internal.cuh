@@ -217,6 +217,7 @@ struct PrefillTcArgs {
     const float* rho0;         // [d] nullable
     bf16 *xe, *xq;             // [pair_cap][d] gathered embedding rows; gamma_1 * u
     float* ssq;                // [ceil(d / 128)][pair_cap]
+    float2* rope;              // [pair_cap][dh / 2] scratch: (cos, sin) at every pair's position
     const int *slot_of, *row_of;
     const double* inv_freq;
     bf16 *Kc, *Vc;

@@ -128,7 +128,7 @@ struct PfParams {
     const bf16* bias;          // [rows] nullable
     int kvw, Hkv, dh, max_len;
     const int *slot_of, *row_of;
-    const double* inv_freq;
+    const float2* rope;        // [pairs][dh / 2] (cos, sin) at the pair's position
     bf16 *Kc, *Vc;
 };
 
@@ -258,9 +258,8 @@ __global__ void __launch_bounds__(PF_THREADS, 1) prefill_tc_kernel(const __grid_
                                 const int ee = e0 + e, f = ee % half;
                                 const int pr = r + e + (ee < half ? half : -half);        // the partner row, in this tile
                                 const float part = mine[pr] * sc + (P.bias ? __bfloat162float(P.bias[row0 + pr]) : 0.f);
-                                float cs, sn;
-                                rope_cs(crow, P.inv_freq[f], cs, sn);
-                                val = ee < half ? val * cs - part * sn : val * cs + part * sn;
+                                const float2 t = __ldg(P.rope + (long long)pair * half + f);
+                                val = ee < half ? val * t.x - part * t.y : val * t.x + part * t.y;
                             }
                             x[e] = val;
                         }
@@ -290,6 +289,17 @@ __global__ void prefill_gather_kernel(const int32_t* ids, int n_pairs, int d, in
         const int n = (int)(i / upr), off = (int)(i % upr);
         const int id = checked_token(ids[n], vocab, id_flag);
         ((uint4*)(xe + (long long)n * d))[off] = ld_stream((const uint4*)(embed + (long long)id * d) + off);
+    }
+}
+
+// (cos, sin) of every pair's position, once per call: every K tile of GEMM 2 rotates with the same angles
+__global__ void prefill_rope_kernel(const int* row_of, int n_pairs, int half, const double* inv_freq, float2* rope) {
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < (long long)n_pairs * half; i += (long long)gridDim.x * blockDim.x) {
+        const int n = (int)(i / half), f = (int)(i % half);
+        const int pos = row_of[n];
+        float cs = 1.f, sn = 0.f;
+        if (pos >= 0) rope_cs(pos, inv_freq[f], cs, sn);
+        rope[i] = make_float2(cs, sn);
     }
 }
 
@@ -347,6 +357,8 @@ cudaError_t launch_prefill_tc(const PrefillTcArgs& a, cudaStream_t st) {
     prefill_gather_kernel<<<592, 256, 0, st>>>(a.ids, a.n_pairs, d, a.vocab, a.embed, a.xe, a.id_flag);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    prefill_rope_kernel<<<296, 256, 0, st>>>(a.row_of, a.n_pairs, a.dh / 2, a.inv_freq, a.rope);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
     PfParams P;
     memset(&P, 0, sizeof(P));
     // ---- GEMM 1: u = W_fc [h ; E[id]] + rho_0
@@ -367,6 +379,6 @@ cudaError_t launch_prefill_tc(const PrefillTcArgs& a, cudaStream_t st) {
     Q.wait_cycles = a.wait_cycles; Q.error_flag = a.error_flag;
     Q.ssq_in = a.ssq; Q.ssq_tiles = (d + PF_TM - 1) / PF_TM; Q.pair_cap = a.pair_cap; Q.d = d; Q.eps = a.eps;
     Q.bias = a.bkv; Q.kvw = a.kvw; Q.Hkv = a.Hkv; Q.dh = a.dh; Q.max_len = a.max_len;
-    Q.slot_of = a.slot_of; Q.row_of = a.row_of; Q.inv_freq = a.inv_freq; Q.Kc = a.Kc; Q.Vc = a.Vc;
+    Q.slot_of = a.slot_of; Q.row_of = a.row_of; Q.rope = a.rope; Q.Kc = a.Kc; Q.Vc = a.Vc;
     return pf_launch<1>(Q, st);
 }
