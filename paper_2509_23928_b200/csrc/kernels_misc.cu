@@ -151,48 +151,60 @@ cudaError_t launch_kv_append(int dtype, const float* kv, int P, const int* slot_
 // ------------------------------------------------------------------------------------------
 // greedy verification in one launch: row argmax over [B][k+1][V], accept length, next token, rollback
 // ------------------------------------------------------------------------------------------
-#define VERIFY_CHUNK 2048   // logits per CTA: one 16-byte load per thread for bf16 logits
+#define VERIFY_MAX_PASSES 8    // 16-byte loads a thread may have in flight
+static_assert(HIVIS_MAX_K + 1 <= 32, "the finishing warp holds one row of a sequence per lane");
 
-// One CTA per (chunk of a row, row, sequence).  Every CTA folds its chunk into the row's packed argmax key
-// (integer max: lowest index among equal values, independent of arrival order) and counts itself on the
-// sequence's arrival counter; the CTA that completes the count reads the sequence's k + 1 keys, finds the
-// longest accepted prefix, writes the outputs, rolls the slot back, and leaves keys and counter zero for the
-// next call.  Nobody waits.
+// One CTA per (chunk of a row, row, sequence); a chunk is `passes` x 256 16-byte vectors, all of a thread's loads
+// issued before the first is used.  Every CTA folds its chunk into the row's packed argmax key (integer max:
+// lowest index among equal values, independent of arrival order) and counts itself on the sequence's arrival
+// counter; the CTA that completes the count reads the sequence's k + 1 keys and k draft ids (one per lane, so the
+// loads overlap), finds the longest accepted prefix, writes the outputs, rolls the slot back, and leaves keys and
+// counter zero for the next call.  Nobody waits.
 template <typename LT>
-__global__ void __launch_bounds__(256) verify_kernel(SlotList sl, int k, const void* logits, int V,
+__global__ void __launch_bounds__(256) verify_kernel(SlotList sl, int k, const void* logits, int V, int passes,
                                                      const int32_t* draft_ids, u64* keys, int* arrivals,
                                                      int* kv_len, int32_t* out_accept, int32_t* out_next,
                                                      int32_t* out_kv_len) {
     __shared__ u64 kred[8];
+    constexpr int VEC = 16 / (int)sizeof(LT);
     const int b = blockIdx.z;
     const long long rowi = (long long)b * (k + 1) + blockIdx.y;
     const LT* row = (const LT*)logits + rowi * V;
-    const int c0 = blockIdx.x * VERIFY_CHUNK;
-    const int c1 = min(V, c0 + VERIFY_CHUNK);
+    const int chunk = passes * 256 * VEC;
+    const int c0 = blockIdx.x * chunk;
+    const int c1 = min(V, c0 + chunk);
     u64 best = 0;
-    constexpr int VEC = 16 / (int)sizeof(LT);
-    const bool aligned = (((size_t)row) & 15) == 0;
+    const bool aligned = (((size_t)(row + c0)) & 15) == 0;
     if (aligned) {
-        const int nvec = (c1 - c0) / VEC;
+        const int nvec = (c1 - c0) / VEC;                 // <= passes * 256
         const uint4* rv = (const uint4*)(row + c0);
-        for (int i = threadIdx.x; i < nvec; i += 256) {
-            const uint4 w = ld_stream(rv + i);
-            const int e0 = c0 + i * VEC;
-            float f[VEC];
-            if constexpr (sizeof(LT) == 2) {
-                f[0] = bf16_lo(w.x); f[1] = bf16_hi(w.x); f[2] = bf16_lo(w.y); f[3] = bf16_hi(w.y);
-                f[4] = bf16_lo(w.z); f[5] = bf16_hi(w.z); f[6] = bf16_lo(w.w); f[7] = bf16_hi(w.w);
-            } else {
-                f[0] = __uint_as_float(w.x); f[1] = __uint_as_float(w.y);
-                f[2] = __uint_as_float(w.z); f[3] = __uint_as_float(w.w);
-            }
+        uint4 w[VERIFY_MAX_PASSES];
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) {
-                const u64 kk = pack_key(f[e], e0 + e);
-                best = kk > best ? kk : best;
+        for (int p = 0; p < VERIFY_MAX_PASSES; ++p) {
+            const int i = threadIdx.x + p * 256;
+            if (i < nvec) w[p] = ld_stream(rv + i);
+        }
+#pragma unroll
+        for (int p = 0; p < VERIFY_MAX_PASSES; ++p) {
+            const int i = threadIdx.x + p * 256;
+            if (i < nvec) {
+                const int e0 = c0 + i * VEC;
+                float f[VEC];
+                if constexpr (sizeof(LT) == 2) {
+                    f[0] = bf16_lo(w[p].x); f[1] = bf16_hi(w[p].x); f[2] = bf16_lo(w[p].y); f[3] = bf16_hi(w[p].y);
+                    f[4] = bf16_lo(w[p].z); f[5] = bf16_hi(w[p].z); f[6] = bf16_lo(w[p].w); f[7] = bf16_hi(w[p].w);
+                } else {
+                    f[0] = __uint_as_float(w[p].x); f[1] = __uint_as_float(w[p].y);
+                    f[2] = __uint_as_float(w[p].z); f[3] = __uint_as_float(w[p].w);
+                }
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) {
+                    const u64 kk = pack_key(f[e], e0 + e);
+                    best = kk > best ? kk : best;
+                }
             }
         }
-        for (int i = c0 + nvec * VEC + threadIdx.x; i < c1; i += 256) {
+        for (int i = c0 + nvec * VEC + threadIdx.x; i < c1; i += 256) {       // V not a multiple of the vector
             const u64 kk = pack_key(load_as_float<LT>(row, i), i);
             best = kk > best ? kk : best;
         }
@@ -209,39 +221,55 @@ __global__ void __launch_bounds__(256) verify_kernel(SlotList sl, int k, const v
     }
     if ((threadIdx.x & 31) == 0) kred[threadIdx.x >> 5] = best;
     __syncthreads();
-    if (threadIdx.x != 0) return;
-    u64 m = kred[0];
+    if (threadIdx.x >= 32) return;
+    const int lane = threadIdx.x;
+    int last = 0;
+    if (lane == 0) {
+        u64 m = kred[0];
 #pragma unroll
-    for (int w = 1; w < 8; ++w) m = kred[w] > m ? kred[w] : m;
-    atomicMax(keys + rowi, m);
-    // release: the key update above is visible before the count; acquire: so are those of earlier arrivers
-    const int total = (int)gridDim.x * (k + 1);
-    if (atom_add_acq_rel(arrivals + b, 1) != total - 1) return;
+        for (int w = 1; w < 8; ++w) m = kred[w] > m ? kred[w] : m;
+        atomicMax(keys + rowi, m);
+        // release: the key update above is visible before the count; acquire: so are those of earlier arrivers
+        const int total = (int)gridDim.x * (k + 1);
+        last = atom_add_acq_rel(arrivals + b, 1) == total - 1;
+    }
+    if (!__shfl_sync(0xffffffffu, last, 0)) return;
+    // lane j holds row j of the sequence: its argmax and the draft token it is compared with
     u64* kr = keys + (long long)b * (k + 1);
-    int n = 0;
-    while (n < k && key_index(__ldcg(kr + n)) == draft_ids[(long long)b * k + n]) ++n;
-    const int next = key_index(__ldcg(kr + n));
     const int slot = sl.slot[b];
-    const int pairs = kv_len[slot] - k + 1;          // true-feature pairs of the sequence
+    const int len = kv_len[slot];
+    const int am = lane <= k ? key_index(__ldcg(kr + lane)) : 0;
+    const int dj = lane < k ? draft_ids[(long long)b * k + lane] : -1;
+    const unsigned miss = __ballot_sync(0xffffffffu, lane < k && am != dj);
+    const int n = miss ? __ffs(miss) - 1 : k;             // length of the accepted prefix
+    const int next = __shfl_sync(0xffffffffu, am, n);
+    if (lane <= k) kr[lane] = 0ull;
+    if (lane != 0) return;
+    const int pairs = len - k + 1;                        // true-feature pairs of the sequence
     const int rows = pairs + (n < k - 1 ? n : k - 1);
     kv_len[slot] = rows;
     out_accept[b] = n;
     out_next[b] = next;
     if (out_kv_len) out_kv_len[b] = rows;
-    for (int j = 0; j <= k; ++j) kr[j] = 0ull;
     arrivals[b] = 0;
 }
 
 cudaError_t launch_verify(int logits_dtype, const SlotList& sl, int k, int V, const int32_t* draft_ids,
                           const void* logits, u64* keys, int* arrivals, int* kv_len, int32_t* out_accept,
                           int32_t* out_next, int32_t* out_kv_len, cudaStream_t st, int* n_launches) {
-    dim3 grid((unsigned)((V + VERIFY_CHUNK - 1) / VERIFY_CHUNK), (unsigned)(k + 1), (unsigned)sl.n);
+    // the shortest chunk that still puts every CTA on the device at once (148 SMs x 8 CTAs of 256 threads)
+    const int per_pass = 256 * (logits_dtype == HIVIS_BF16 ? 8 : 4);
+    const long long rows = (long long)sl.n * (k + 1);
+    int passes = 1;
+    while (passes < VERIFY_MAX_PASSES && rows * ((V + passes * per_pass - 1) / (passes * per_pass)) > 148 * 8) ++passes;
+    const int chunk = passes * per_pass;
+    dim3 grid((unsigned)((V + chunk - 1) / chunk), (unsigned)(k + 1), (unsigned)sl.n);
     if (logits_dtype == HIVIS_BF16)
-        verify_kernel<bf16><<<grid, 256, 0, st>>>(sl, k, logits, V, draft_ids, keys, arrivals, kv_len, out_accept,
-                                                   out_next, out_kv_len);
+        verify_kernel<bf16><<<grid, 256, 0, st>>>(sl, k, logits, V, passes, draft_ids, keys, arrivals, kv_len,
+                                                   out_accept, out_next, out_kv_len);
     else
-        verify_kernel<float><<<grid, 256, 0, st>>>(sl, k, logits, V, draft_ids, keys, arrivals, kv_len, out_accept,
-                                                    out_next, out_kv_len);
+        verify_kernel<float><<<grid, 256, 0, st>>>(sl, k, logits, V, passes, draft_ids, keys, arrivals, kv_len,
+                                                    out_accept, out_next, out_kv_len);
     *n_launches = 1;
     return cudaGetLastError();
 }
