@@ -510,6 +510,97 @@ def prefill_ablation(reps: int = 5):
     return out
 
 
+def tree_and_sampling(weights: WeightCache, reps: int = 30):
+    """The two widened rows, timed with CUDA events around the calls (medians of `reps`, caches warm as in a running
+    decode loop; between tree drafts the target logits of the previous verification are rewritten, 23 MB):
+    tree drafting and greedy tree verification of one sequence of the headline workload with the paper's tree shapes
+    (top-10, depth 6, 60 kept; top-8, depth 4, 30 kept), and verification by speculative sampling at batch 16.
+    Algorithmic bytes of a tree draft: every level streams the drafter's weights once and reads the prefix rows of the
+    cache once per expanded node."""
+    import torch
+    from hivis_inputs.device import to_dev
+    from paper_2509_23928_b200 import Drafter
+    peak, peak_kind = measured_peaks()
+    out = {"unit": "us", "peak_GBps": peak, "peak_kind": peak_kind, "trees": [], "launches": reps}
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    wl = hi.workload(HEADLINE)
+    ids, hidden, cu = hi.make_prompt(wl)
+    resid = hi.make_residuals(wl)
+    T = int(cu[1])
+    D = wl.dims
+    es = 2 if D.dtype == "bf16" else 4
+    dr = Drafter(D, weights.get(wl), max_batch=1, max_len=T + 80, max_k=8)
+    d_resid = to_dev(resid, D.dtype)
+    dr.prefill(torch.from_numpy(ids).cuda(), to_dev(hidden, D.dtype), [int(x) for x in cu], resid0=d_resid[0])
+    weight_bytes = dr.step_bytes([0]) - 2 * D.kv_dim * es               # one position with an empty prefix: the weights
+    rng = np.random.default_rng(7)
+    for topk, depth, keep in ((10, 6, 60), (8, 4, 30)):
+        logits = to_dev(rng.standard_normal((keep + 1, D.vocab)).astype(np.float32), wl.logits_dtype)
+        d_ms, v_ms = [], []
+        n0 = dr.launch_count()
+        for i in range(reps + 3):
+            dr.set_kv_len(0, T - 1, restore_pending=True)
+            a, b, c = ev(), ev(), ev()
+            a.record()
+            tok, par, sc, cnt = dr.draft_tree(0, topk, depth, keep, d_resid)
+            b.record()
+            dr.verify_tree(0, depth, logits)
+            c.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                d_ms.append(a.elapsed_time(b)); v_ms.append(b.elapsed_time(c))
+        launches = (dr.launch_count() - n0) / (reps + 3) - 1            # the restore kernel
+        nodes = 1 + (depth - 1) * topk                                   # positions that run through the layer
+        nbytes = depth * weight_bytes + nodes * 2 * (T - 1) * D.kv_dim * es
+        us = float(np.median(d_ms)) * 1e3
+        out["trees"].append({"workload": wl.name, "topk": topk, "depth": depth, "keep": keep, "kept": int(cnt[0].item()),
+                             "draft_tree_us": round(us, 1), "verify_tree_us": round(float(np.median(v_ms)) * 1e3, 1),
+                             "launches_per_tree": round(launches, 1), "layer_positions": nodes,
+                             "algorithmic_bytes": int(nbytes), "GBps": round(nbytes / (us * 1e-6) / 1e9, 1),
+                             "frac_of_peak": round(nbytes / (us * 1e-6) / 1e9 / peak, 4)})
+    dr.status()
+    dr.close()
+
+    wl = hi.workload(BATCH16)
+    B, k, V = wl.batch, wl.k, wl.dims.vocab
+    ids, hidden, cu = hi.make_prompt(wl)
+    lens = np.diff(cu)
+    resid = hi.make_residuals(wl)
+    dr = Drafter(wl.dims, weights.get(wl), max_batch=B, max_len=int(lens.max()) + k + 8, max_k=8)
+    d_resid = to_dev(resid, wl.dims.dtype)
+    dr.prefill(torch.from_numpy(ids).cuda(), to_dev(hidden, wl.dims.dtype), [int(x) for x in cu], resid0=d_resid[0])
+    out_ids, d_logits = dr.draft(B, k, d_resid, want_logits=True)
+    target = to_dev(rng.standard_normal((B, k + 1, V)).astype(np.float32), wl.logits_dtype)
+    ua = torch.from_numpy(rng.random((B, k)).astype(np.float32)).cuda()
+    us_ = torch.from_numpy(rng.random(B).astype(np.float32)).cuda()
+    flush = torch.empty(160 << 20, dtype=torch.uint8, device="cuda")
+    t_ms = []
+    for i in range(reps + 3):
+        for b in range(B):
+            dr.set_kv_len(b, int(lens[b]) - 1, restore_pending=True)
+        dr.draft(B, k, d_resid, out_ids=out_ids)
+        flush.zero_()                                                    # the logits come from DRAM
+        a, b_ = ev(), ev()
+        a.record()
+        dr.verify_sampled(out_ids, d_logits, target, 1.0, ua, us_)
+        b_.record()
+        torch.cuda.synchronize()
+        if i >= 3:
+            t_ms.append(a.elapsed_time(b_))
+    tb = 2 if wl.logits_dtype == "bf16" else 4
+    # every logit once for the row statistics, then per sequence the target and draft rows at the first rejection
+    lbytes = B * k * V * 4 + B * (k + 1) * V * tb + B * V * (4 + tb)
+    us = float(np.median(t_ms)) * 1e3
+    out["sampled_verification"] = {"workload": wl.name, "batch": B, "k": k, "vocab": V, "temperature": 1.0,
+                                   "us": round(us, 1), "launches": 2, "algorithmic_bytes": int(lbytes),
+                                   "GBps": round(lbytes / (us * 1e-6) / 1e9, 1),
+                                   "frac_of_peak": round(lbytes / (us * 1e-6) / 1e9 / peak, 4)}
+    dr.status()
+    dr.close()
+    return out
+
+
 def stub_replica(rank: int) -> dict:
     """Stands in for the device work when HIVIS_BENCH_STUB=1 (CPU test of the launch path only): fixed fake
     times, rank 1 slower.  The line it leads to is marked as a stub and carries no measurement."""
@@ -529,6 +620,8 @@ def main():
                     help="mask of weight matrices the tensor-core chain kernel asks L2 to keep (HIVIS_OPT_L2_KEEP; study aid)")
     ap.add_argument("--prefill-ablation", action="store_true",
                     help="time the prefix build with 0 / 576 / 2048 leading (visual stand-in) positions and exit")
+    ap.add_argument("--tree-and-sampling", action="store_true",
+                    help="time tree drafting + tree verification (one sequence) and speculative-sampling verification (batch 16)")
     ap.add_argument("--phase-times", action="store_true",
                     help="print where a draft step of the tensor-core chain kernel goes (its own time stamps) and exit")
     args = ap.parse_args()
@@ -584,6 +677,9 @@ def main():
     weights = WeightCache()
     if args.prefill_ablation:
         print(json.dumps(prefill_ablation()))
+        return
+    if args.tree_and_sampling:
+        print(json.dumps(tree_and_sampling(weights)))
         return
     if args.phase_times:
         print(json.dumps(phase_breakdown(hi.workload(args.workload or BATCH16), weights)))

@@ -30,7 +30,7 @@ struct hivis_ctx {
     bf16 *feat_h, *xq, *attn_h, *xm, *act_h;
     u64* keys;
     int key_stride;
-    float2* vstats;               // sampled verification: (max, log sum exp) of every logits row [max_batch * (2 max_k + 1)]
+    float2* vstats;               // sampled verification: (max, sum exp) of every piece of every logits row
     u64* vkeys;                   // verification: argmax keys [max_batch][max_k + 1] and arrival counters
     int* varrive;                 // [max_batch]; both zero between calls
     float *part_acc, *part_ml;
@@ -317,7 +317,7 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
          dalloc(c, &c->rho, (long long)HIVIS_MAX_K * d) && dalloc(c, &c->ssq1, tiles1 * R) &&
          dalloc(c, &c->ssq2, tiles1 * R) && dalloc(c, &c->keys, R * c->key_stride) &&
          dalloc(c, &c->vkeys, MB * (cfg->max_k + 1)) && dalloc(c, &c->varrive, MB) &&
-         dalloc(c, &c->vstats, MB * (2 * cfg->max_k + 1)) &&
+         dalloc(c, &c->vstats, (long long)sampled_stats_entries(cfg->max_batch, cfg->max_k, cfg->vocab)) &&
          dalloc(c, &c->part_acc, R * cfg->n_q_heads * (long long)c->nsplit_cap * cfg->head_dim) &&
          dalloc(c, &c->part_ml, R * cfg->n_q_heads * (long long)c->nsplit_cap * 2) &&
          dalloc(c, &c->counters, R * cfg->n_q_heads) && dalloc(c, &c->bar_counter, 1) &&
@@ -679,6 +679,38 @@ int hivis_prefill(hivis_ctx* c, int B, const int* seq_slots_host, const int32_t*
     return HIVIS_OK;
 }
 
+// Arguments of the tensor-core chain kernel for B columns and k steps (the whole step; callers narrow seq_first /
+// seq_last and bar_base when they run a part of it).
+static void fill_tc_args(hivis_ctx* c, TcArgs* out, int B, int k, int lo, const float* rho, int n_resid,
+                         const int32_t* forced_ids, float* out_logits) {
+    const hivis_config& g = c->cfg;
+    ChainArgs ca;
+    fill_chain_args(c, &ca);
+    TcArgs& a = *out;
+    memset(&a, 0, sizeof(a));
+    for (int p = 0; p < PH_COUNT; ++p) a.ph[p] = ca.ph[p];
+    a.k = k; a.B = B; a.lo = lo;
+    a.d = g.d; a.qw = c->qw; a.kvw = c->kvw; a.F = g.ffn; a.V = g.vocab; a.Hq = g.n_q_heads; a.Hkv = g.n_kv_heads;
+    a.dh = g.head_dim; a.max_len = g.max_len; a.eps = g.rms_eps; a.scale = 1.0f / sqrtf((float)g.head_dim);
+    a.norm1 = (const bf16*)c->norm1; a.norm2 = (const bf16*)c->norm2; a.bqkv = (const bf16*)c->bqkv;
+    a.rho = rho; a.n_resid = n_resid;
+    a.slots = c->d_slots; a.pos0 = c->d_pos0; a.cur_id = c->cur_id; a.forced = forced_ids;
+    a.keys = c->keys; a.key_stride = c->key_stride;
+    a.u = c->u; a.qkv = c->qkv; a.attn = c->attn; a.y = c->y; a.feat = c->feat;
+    a.feat_h = c->feat_h; a.xq_h = c->xq; a.attn_h = c->attn_h; a.xm_h = c->xm; a.act_h = c->act_h;
+    a.xe_h = c->xe_h; a.embed = (const bf16*)c->embed; a.rope_tab = c->rope_tab;
+    a.ssq1 = c->ssq1; a.ssq2 = c->ssq2; a.logits_out = out_logits;
+    a.partial = c->tc_partial; a.tile_ctr = c->tile_ctr;
+    a.Kc = c->Kc; a.Vc = c->Vc; a.inv_freq = c->inv_freq; a.part_acc = c->part_acc; a.part_ml = c->part_ml;
+    a.counters = c->counters;
+    a.attn_nslot = c->nsplit_cap;
+    a.bar_counter = c->bar_counter; a.bar_base = c->bar_count_host + (c->debug_skew ? (1ull << 40) : 0ull);
+    a.wait_cycles = c->wait_cycles; a.error_flag = c->error_flag; a.id_flag = c->id_flag;
+    a.l2_keep = c->opt_l2_keep;
+    a.phase_t = nullptr;
+    a.seq_first = 0; a.seq_last = 7;
+}
+
 int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const void* resid, int n_resid,
                 int32_t* out_ids, const int32_t* forced_ids, float* out_logits, void* stream) {
     if (!c) return HIVIS_ERR_ARG;
@@ -737,30 +769,8 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
         CKP(c, CLS_OTHER, st, launch_tc_setup(sl, k, d, lo, c->d_slots, c->d_pos0, c->kv_len, c->pend_feat, c->pend_id,
                                               c->feat, c->feat_h, c->cur_id, c->keys, c->key_stride, (const bf16*)c->embed,
                                               V, c->xe_h, c->id_flag, st));
-        ChainArgs ca;
-        fill_chain_args(c, &ca);
         TcArgs a;
-        memset(&a, 0, sizeof(a));
-        for (int p = 0; p < PH_COUNT; ++p) a.ph[p] = ca.ph[p];
-        a.k = k; a.B = B; a.lo = lo;
-        a.d = d; a.qw = c->qw; a.kvw = c->kvw; a.F = F; a.V = V; a.Hq = g.n_q_heads; a.Hkv = g.n_kv_heads;
-        a.dh = g.head_dim; a.max_len = g.max_len; a.eps = g.rms_eps; a.scale = 1.0f / sqrtf((float)g.head_dim);
-        a.norm1 = (const bf16*)c->norm1; a.norm2 = (const bf16*)c->norm2; a.bqkv = (const bf16*)c->bqkv;
-        a.rho = resid ? c->rho : nullptr; a.n_resid = resid ? n_resid : 1;
-        a.slots = c->d_slots; a.pos0 = c->d_pos0; a.cur_id = c->cur_id; a.forced = forced_ids;
-        a.keys = c->keys; a.key_stride = c->key_stride;
-        a.u = c->u; a.qkv = c->qkv; a.attn = c->attn; a.y = c->y; a.feat = c->feat;
-        a.feat_h = c->feat_h; a.xq_h = c->xq; a.attn_h = c->attn_h; a.xm_h = c->xm; a.act_h = c->act_h;
-        a.xe_h = c->xe_h; a.embed = (const bf16*)c->embed; a.rope_tab = c->rope_tab;
-        a.ssq1 = c->ssq1; a.ssq2 = c->ssq2; a.logits_out = out_logits;
-        a.partial = c->tc_partial; a.tile_ctr = c->tile_ctr;
-        a.Kc = c->Kc; a.Vc = c->Vc; a.inv_freq = c->inv_freq; a.part_acc = c->part_acc; a.part_ml = c->part_ml;
-        a.counters = c->counters;
-        a.attn_nslot = c->nsplit_cap;
-        a.bar_counter = c->bar_counter; a.bar_base = c->bar_count_host + (c->debug_skew ? (1ull << 40) : 0ull);
-        a.wait_cycles = c->wait_cycles; a.error_flag = c->error_flag; a.id_flag = c->id_flag;
-        a.l2_keep = c->opt_l2_keep;
-        a.phase_t = nullptr;
+        fill_tc_args(c, &a, B, k, lo, resid ? c->rho : nullptr, resid ? n_resid : 1, forced_ids, out_logits);
         if (c->opt_phase_times) {
             CK(c, cudaMemsetAsync(c->phase_t, 0, (size_t)k * HIVIS_PHASE_EVENTS * c->num_sms * sizeof(u64), st));
             a.phase_t = c->phase_t;
@@ -923,21 +933,44 @@ int hivis_draft_tree(hivis_ctx* c, int slot, int topk, int depth, int keep, cons
     }
     const TreeBufs& T = c->tree;
     CKL(c, launch_tree_begin(slot, d, c->kv_len, c->pend_feat, c->pend_id, c->feat, c->feat_h, c->cur_id, c->d_slots, T, st));
+    // bf16 drafters with up to 16 nodes per level (always, by the limit on topk) run the levels' GEMMs in the
+    // tensor-core chain kernel, one step long and in two parts around the tree's own attention
+    const bool tc = c->tc_ok && c->opt_tc != 0;
     for (int level = 0; level < depth; ++level) {
         const int nb = level == 0 ? 1 : topk;
-        const bool mma = use_mma(c, nb, false);
         if (level > 0) CKL(c, launch_tree_gather(nb, d, c->tree_g, T, c->feat, c->feat_h, c->cur_id, st));
         const int row = level < n_resid - 1 ? level : n_resid - 1;
         const float* rho = resid ? c->rho + (long long)row * d : nullptr;
-        rc = run_fuse(c, mma, 0, nb, c->feat, c->feat_h, c->cur_id, 1, nullptr, rho, st);
-        if (rc) return rc;
-        rc = run_qkv(c, mma, 0, nb, 0, c->qkvw, c->qkv, st);
-        if (rc) return rc;
-        CK(c, launch_tree_attention(c->dtype, nb, c->qkv, c->qkvw, g.n_q_heads, g.n_kv_heads, g.head_dim, g.max_len, slot,
-                                    level, T, c->inv_freq, c->Kc, c->Vc, c->attn, c->attn_h, st));
-        c->launches += 2;
-        rc = run_after_attention(c, mma, 0, nb, c->keys, c->key_stride, c->tree_logits, V, st);
-        if (rc) return rc;
+        if (tc) {
+            const int lo = tc_lo_offset(nb);
+            const u64 G = (u64)c->num_sms;
+            CKL(c, launch_tree_operands_tc(nb, TC_OP_ROWS, d, lo, c->feat, c->cur_id, (const bf16*)c->embed, V, c->feat_h,
+                                           c->xe_h, c->d_pos0, c->id_flag, st));
+            TcArgs a;
+            fill_tc_args(c, &a, nb, 1, lo, rho, 1, nullptr, c->tree_logits);
+            a.seq_first = 0; a.seq_last = 2;                         // gather, fusion FC, QKV
+            c->debug_skew = false;
+            CKL(c, launch_tc_chain(c->tc_maps, a, c->num_sms, st));
+            c->bar_count_host += G * 3;
+            CK(c, launch_tree_attention(c->dtype, nb, c->qkv, c->qkvw, g.n_q_heads, g.n_kv_heads, g.head_dim, g.max_len, slot,
+                                        level, T, c->inv_freq, c->Kc, c->Vc, c->attn, c->attn_h, lo, st));
+            c->launches += 2;
+            a.seq_first = 4; a.seq_last = 7;                         // O, gate/up, down, LM head (logits of every node)
+            a.bar_base = c->bar_count_host - G * 4;                  // as if gather .. attention had been arrived on
+            CKL(c, launch_tc_chain(c->tc_maps, a, c->num_sms, st));
+            c->bar_count_host += G * 4;
+        } else {
+            const bool mma = use_mma(c, nb, false);
+            rc = run_fuse(c, mma, 0, nb, c->feat, c->feat_h, c->cur_id, 1, nullptr, rho, st);
+            if (rc) return rc;
+            rc = run_qkv(c, mma, 0, nb, 0, c->qkvw, c->qkv, st);
+            if (rc) return rc;
+            CK(c, launch_tree_attention(c->dtype, nb, c->qkv, c->qkvw, g.n_q_heads, g.n_kv_heads, g.head_dim, g.max_len, slot,
+                                        level, T, c->inv_freq, c->Kc, c->Vc, c->attn, c->attn_h, 0, st));
+            c->launches += 2;
+            rc = run_after_attention(c, mma, 0, nb, c->keys, c->key_stride, c->tree_logits, V, st);
+            if (rc) return rc;
+        }
         CKL(c, launch_tree_topk(nb, c->tree_logits, V, topk, T, st));
         CK(c, cudaMemcpyAsync(c->tree_g, c->feat, (size_t)nb * d * sizeof(float), cudaMemcpyDeviceToDevice, st));
         CKL(c, launch_tree_select(level, depth, nb, topk, T, st));

@@ -189,6 +189,10 @@ struct TcArgs {
     int* id_flag;              // set non-zero when a token id outside [0, V) reached the embedding lookup
     u64* phase_t;              // nullable: [k][HIVIS_PHASE_EVENTS][grid] time stamps (HIVIS_OPT_PHASE_TIMES)
     int l2_keep;               // bit p set: the weights of phase p are loaded with the keep-in-L2 policy
+    // The grid barriers of a step are numbered 0 gather, 1 FC, 2 QKV, 3 attention, 4 O, 5 gate/up, 6 down, 7 LM head.
+    // A launch runs the part [seq_first, seq_last] of every step (0..7: the whole step); what lies outside does no work
+    // and arrives nowhere, and bar_base is set as if the barriers before seq_first had been completed already.
+    int seq_first, seq_last;
 };
 // fills `maps` for the given buffers; returns cudaSuccess or an error (driver entry point missing, bad shape)
 cudaError_t tc_build_maps(TcMaps* maps, const ChainPhase* ph, int d, int qw, int F, const bf16* feat_h,
@@ -254,7 +258,12 @@ cudaError_t launch_tree_gather(int nb, int d, const float* g_prev, const TreeBuf
                                cudaStream_t st);
 cudaError_t launch_tree_attention(int dtype, int nb, const float* qkv, int ld, int Hq, int Hkv, int dh, int max_len,
                                   int slot, int level, const TreeBufs& T, const double* inv_freq, void* Kc, void* Vc,
-                                  float* attn, bf16* attn_h, cudaStream_t st);
+                                  float* attn, bf16* attn_h, int lo_rows, cudaStream_t st);
+// the level's rows as the tensor-core chain kernel reads them (`rows` = all operand rows, so that those beyond the
+// level are cleared)
+cudaError_t launch_tree_operands_tc(int nb, int rows, int d, int lo_rows, const float* feat, const int* cur_id,
+                                    const bf16* embed, int vocab, bf16* feat_h, bf16* xe_h, int* pos0, int* id_flag,
+                                    cudaStream_t st);
 cudaError_t launch_tree_topk(int nb, const float* logits, int V, int topk, const TreeBufs& T, cudaStream_t st);
 cudaError_t launch_tree_select(int level, int depth, int nb, int topk, const TreeBufs& T, cudaStream_t st);
 cudaError_t launch_tree_finalize(int keep, const TreeBufs& T, int32_t* out_tokens, int32_t* out_parents, float* out_scores,
@@ -299,7 +308,8 @@ cudaError_t launch_verify(int logits_dtype, const SlotList& sl, int k, int V, co
                           int32_t* out_next, int32_t* out_kv_len, cudaStream_t st, int* n_launches);
 
 // verification by speculative sampling: per-row softmax statistics, then acceptance tests, the draw of the next token
-// and the rollback; stats: [B * (2k + 1)] scratch
+// and the rollback; stats: scratch of sampled_stats_entries(max_batch, max_k, V) entries (one per piece of a row)
+int sampled_stats_entries(int max_batch, int max_k, int V);
 cudaError_t launch_verify_sampled(int logits_dtype, const SlotList& sl, int k, int V, float temperature,
                                   const int32_t* draft_ids, const float* draft_logits, const void* target_logits,
                                   float2* stats, const float* u_accept, const float* u_sample, int* kv_len,

@@ -4,68 +4,93 @@
 // (from p of the last row when every token was kept).  The uniform numbers come from the caller.
 #include "attn_body.cuh"
 
-__device__ __forceinline__ float sblock_max(float v, float* red) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
-    __syncthreads();
-    float r = red[0];
-    for (int w = 1; w < 8; ++w) r = fmaxf(r, red[w]);
-    return r;
-}
-__device__ __forceinline__ double sblock_sum(double v, double* red) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
-    __syncthreads();
-    double r = 0.0;
-    for (int w = 0; w < 8; ++w) r += red[w];
-    return r;
-}
+#define SV_SPAN 4096            // logits of a row that one CTA of the statistics kernel covers (16 per thread, kept in registers)
+#define SV_THREADS 1024         // threads per sequence in the decision kernel
+#define SV_CHUNK 1024           // tokens per chunk of the inverse CDF (one warp sums a chunk)
+#define SV_MAX_CHUNKS 1024
 
-// One CTA per logits row: its maximum and the logarithm of the sum of exp((x - max) / T).
+// Pieces of a row: piece c covers logits [c * SV_SPAN, min(V, (c + 1) * SV_SPAN)).
+__host__ __device__ __forceinline__ int sv_pieces(int V) { return (V + SV_SPAN - 1) / SV_SPAN; }
+
+// One CTA per piece of a logits row: its maximum and the sum of exp((x - max) / T), each logit read once.
 // Rows [0, n_target) are the target's (type LT), rows [n_target, n_target + n_draft) the drafter's (fp32).
 template <typename LT>
 __global__ void __launch_bounds__(256) row_stats_kernel(const void* target, const float* draft, int n_target, int V,
-                                                        float inv_t, float2* stats) {
+                                                        float inv_t, float2* part) {
     __shared__ float redf[8];
-    __shared__ double redd[8];
-    const int r = blockIdx.x;
+    const int r = blockIdx.y, c0 = blockIdx.x * SV_SPAN;
     const bool is_t = r < n_target;
     const LT* tr = (const LT*)target + (long long)r * V;
     const float* dr = draft + (long long)(r - n_target) * V;
+    float x[SV_SPAN / 256];
     float mx = -INFINITY;
-    for (int i = threadIdx.x; i < V; i += 256) mx = fmaxf(mx, is_t ? load_as_float<LT>(tr, i) : dr[i]);
-    mx = sblock_max(mx, redf);
+#pragma unroll
+    for (int j = 0; j < SV_SPAN / 256; ++j) {
+        const int i = c0 + j * 256 + threadIdx.x;
+        x[j] = i < V ? (is_t ? load_as_float<LT>(tr, i) : __ldg(dr + i)) : -INFINITY;
+        mx = fmaxf(mx, x[j]);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if ((threadIdx.x & 31) == 0) redf[threadIdx.x >> 5] = mx;
+    __syncthreads();
+    mx = redf[0];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) mx = fmaxf(mx, redf[w]);
+    __syncthreads();
+    float se = 0.f;
+#pragma unroll
+    for (int j = 0; j < SV_SPAN / 256; ++j) se += expf((x[j] - mx) * inv_t);         // exp(-inf) = 0 beyond the row
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
+    if ((threadIdx.x & 31) == 0) redf[threadIdx.x >> 5] = se;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) t += (double)redf[w];
+        part[(long long)r * gridDim.x + blockIdx.x] = make_float2(mx, (float)t);
+    }
+}
+
+// (max, log sum exp((x - max) / T)) of a row from its pieces
+__device__ __forceinline__ float2 sv_row_stats(const float2* part, int pieces, float inv_t) {
+    float mx = -INFINITY;
+    for (int c = 0; c < pieces; ++c) mx = fmaxf(mx, part[c].x);
     double se = 0.0;
-    for (int i = threadIdx.x; i < V; i += 256) se += (double)expf(((is_t ? load_as_float<LT>(tr, i) : dr[i]) - mx) * inv_t);
-    se = sblock_sum(se, redd);
-    if (threadIdx.x == 0) stats[r] = make_float2(mx, (float)log(se));
+    for (int c = 0; c < pieces; ++c) se += (double)part[c].y * (double)expf((part[c].x - mx) * inv_t);
+    return make_float2(mx, (float)log(se));
 }
 
 // One CTA per sequence: acceptance tests, then the draw of the next token by inverse CDF, then the rollback.
+// The masses of the row that is drawn from are summed per chunk of 1024 tokens (a warp per chunk, fixed order), the
+// chunk that holds u * total is found from the chunk sums and only that chunk is scanned.
 template <typename LT>
-__global__ void __launch_bounds__(256) sampled_verify_kernel(SlotList sl, int k, int V, float inv_t, const int32_t* draft_ids,
-                                                             const float* draft, const void* target, const float2* stats,
-                                                             const float* u_accept, const float* u_sample, int* kv_len,
-                                                             int32_t* out_accept, int32_t* out_next, int32_t* out_kv_len) {
-    __shared__ int s_acc[HIVIS_MAX_K], s_n, s_found;
-    __shared__ double redd[8];
-    __shared__ float s_warp[8];
-    __shared__ double s_base;
-    const int b = blockIdx.x, tid = threadIdx.x, B = sl.n;
-    const float2* st_t = stats + (long long)b * (k + 1);
-    const float2* st_d = stats + (long long)B * (k + 1) + (long long)b * k;
+__global__ void __launch_bounds__(SV_THREADS) sampled_verify_kernel(SlotList sl, int k, int V, float inv_t,
+                                                                    const int32_t* draft_ids, const float* draft,
+                                                                    const void* target, const float2* part,
+                                                                    const float* u_accept, const float* u_sample, int* kv_len,
+                                                                    int32_t* out_accept, int32_t* out_next,
+                                                                    int32_t* out_kv_len) {
+    __shared__ float2 s_st[2 * HIVIS_MAX_K + 1];      // rows 0..k: the target's, k+1..2k: the drafter's
+    __shared__ int s_acc[HIVIS_MAX_K], s_n, s_found, s_chunk, s_clast, s_last[SV_THREADS / 32];
+    __shared__ double s_sum[SV_MAX_CHUNKS], s_base, s_tot;
+    __shared__ float s_warp[SV_THREADS / 32];
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, B = sl.n;
+    const int pieces = sv_pieces(V);
+    if (tid < 2 * k + 1) {
+        const long long row = tid <= k ? (long long)b * (k + 1) + tid : (long long)B * (k + 1) + (long long)b * k + (tid - k - 1);
+        s_st[tid] = sv_row_stats(part + row * pieces, pieces, inv_t);
+    }
+    __syncthreads();
     if (tid < k) {
         const int x = draft_ids[(long long)b * k + tid];
         const LT* tr = (const LT*)target + ((long long)b * (k + 1) + tid) * V;
         const float* dr = draft + ((long long)b * k + tid) * V;
         int ok = 0;
         if (x >= 0 && x < V) {
-            const float lp = (load_as_float<LT>(tr, x) - st_t[tid].x) * inv_t - st_t[tid].y;
-            const float lq = (dr[x] - st_d[tid].x) * inv_t - st_d[tid].y;
+            const float lp = (load_as_float<LT>(tr, x) - s_st[tid].x) * inv_t - s_st[tid].y;
+            const float lq = (dr[x] - s_st[k + 1 + tid].x) * inv_t - s_st[k + 1 + tid].y;
             const float a = expf(fminf(0.f, lp - lq));
             ok = u_accept[(long long)b * k + tid] < a ? 1 : 0;
         }
@@ -77,54 +102,91 @@ __global__ void __launch_bounds__(256) sampled_verify_kernel(SlotList sl, int k,
         while (n < k && s_acc[n]) ++n;
         s_n = n;
         s_found = V;
-        s_base = 0.0;
+        s_clast = -1;
     }
     __syncthreads();
     const int n = s_n;
     const LT* tr = (const LT*)target + ((long long)b * (k + 1) + n) * V;
     const float* dr = draft + ((long long)b * k + (n < k ? n : 0)) * V;
-    const float mt = st_t[n].x, lt = st_t[n].y;
-    const float md = n < k ? st_d[n].x : 0.f, ld = n < k ? st_d[n].y : 0.f;
-    auto pmass = [&](int i) { return expf((load_as_float<LT>(tr, i) - mt) * inv_t - lt); };
+    const float mt = s_st[n].x, lt = s_st[n].y;
+    const float md = n < k ? s_st[k + 1 + n].x : 0.f, ld = n < k ? s_st[k + 1 + n].y : 0.f;
     auto mass = [&](int i, bool resid) {
-        const float p = pmass(i);
+        const float p = expf((load_as_float<LT>(tr, i) - mt) * inv_t - lt);
         if (!resid) return p;
-        const float q = expf((dr[i] - md) * inv_t - ld);
+        const float q = expf((__ldg(dr + i) - md) * inv_t - ld);
         return fmaxf(p - q, 0.f);
     };
+    const int nchunks = (V + SV_CHUNK - 1) / SV_CHUNK;
     bool resid = n < k;
-    double tot = 0.0;
-    for (int i = tid; i < V; i += 256) tot += (double)mass(i, resid);
-    tot = sblock_sum(tot, redd);
-    if (resid && !(tot > 0.0)) {            // p == q exactly: nothing is left over (and such a token is never rejected)
-        resid = false;
-        tot = 0.0;
-        for (int i = tid; i < V; i += 256) tot += (double)pmass(i);
-        tot = sblock_sum(tot, redd);
-    }
-    const double want = (double)u_sample[b] * tot;
-    // inverse CDF: chunks of 256 x 4 consecutive tokens, an exclusive scan inside the chunk, a running base across chunks
     int last_pos = -1;
-    for (int c0 = 0; c0 < V && s_found == V; c0 += 1024) {
-        float m[4];
-        float loc = 0.f;
+    for (int pass = 0; pass < 2; ++pass) {
+        // chunk sums: lane l of the chunk's warp takes tokens 4 l .. 4 l + 3 of every 128
+        last_pos = -1;
+        for (int c = warp; c < nchunks; c += SV_THREADS / 32) {
+            double acc = 0.0;
+#pragma unroll
+            for (int j = 0; j < SV_CHUNK / 128; ++j) {
+                float loc = 0.f;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int i = c * SV_CHUNK + j * 128 + lane * 4 + e;
+                    const float m = i < V ? mass(i, resid) : 0.f;
+                    if (m > 0.f) last_pos = i;
+                    loc += m;
+                }
+                acc += (double)loc;
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            if (lane == 0) s_sum[c] = acc;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            double tot = 0.0;
+            for (int c = 0; c < nchunks; ++c) tot += s_sum[c];
+            s_tot = tot;
+        }
+        __syncthreads();
+        // p == q exactly: nothing is left over (and such a token is never rejected): draw from p
+        if (!(resid && !(s_tot > 0.0))) break;
+        __syncthreads();
+        resid = false;
+    }
+    const double want = (double)u_sample[b] * s_tot;
+    if (tid == 0) {
+        double run = 0.0;
+        int c = 0;
+        for (; c < nchunks - 1; ++c) {
+            if (run + s_sum[c] > want) break;
+            run += s_sum[c];
+        }
+        s_chunk = c;
+        s_base = run;
+    }
+    __syncthreads();
+    {
+        // the chunk that holds the wanted mass: four consecutive tokens per thread, an exclusive scan over the block
+        const int c0 = s_chunk * SV_CHUNK;
+        float m[4], loc = 0.f;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const int i = c0 + tid * 4 + e;
-            m[e] = i < V ? mass(i, resid) : 0.f;
-            if (m[e] > 0.f) last_pos = i;
+            m[e] = (tid < SV_CHUNK / 4 && i < V) ? mass(i, resid) : 0.f;
             loc += m[e];
         }
-        float incl = loc;                   // inclusive scan over the warp
+        // (should rounding keep the scan below the wanted mass although the chunk sums said it is here: the chunk's
+        // last token with mass)
+        if (loc > 0.f) atomicMax(&s_clast, c0 + tid * 4 + (m[3] > 0.f ? 3 : m[2] > 0.f ? 2 : m[1] > 0.f ? 1 : 0));
+        float incl = loc;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const float t = __shfl_up_sync(0xffffffffu, incl, o);
-            if ((tid & 31) >= o) incl += t;
+            if (lane >= o) incl += t;
         }
-        if ((tid & 31) == 31) s_warp[tid >> 5] = incl;
+        if (lane == 31) s_warp[warp] = incl;
         __syncthreads();
         float wbase = 0.f;
-        for (int w = 0; w < (tid >> 5); ++w) wbase += s_warp[w];
+        for (int w = 0; w < warp; ++w) wbase += s_warp[w];
         double run = s_base + (double)wbase + (double)(incl - loc);
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -134,20 +196,16 @@ __global__ void __launch_bounds__(256) sampled_verify_kernel(SlotList sl, int k,
                 break;
             }
         }
-        __syncthreads();
-        if (tid == 255) s_base += (double)wbase + (double)incl;
-        __syncthreads();
     }
     // rounding may leave the cumulative sum a hair below u * total: the last token with mass
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) last_pos = max(last_pos, __shfl_xor_sync(0xffffffffu, last_pos, o));
-    __shared__ int s_last[8];
-    if ((tid & 31) == 0) s_last[tid >> 5] = last_pos;
+    if (lane == 0) s_last[warp] = last_pos;
     __syncthreads();
     if (tid == 0) {
         int lp = s_last[0];
-        for (int w = 1; w < 8; ++w) lp = max(lp, s_last[w]);
-        const int next = s_found < V ? s_found : (lp >= 0 ? lp : 0);
+        for (int w = 1; w < SV_THREADS / 32; ++w) lp = max(lp, s_last[w]);
+        const int next = s_found < V ? s_found : (s_chunk < nchunks - 1 && s_clast >= 0) ? s_clast : (lp >= 0 ? lp : 0);
         const int slot = sl.slot[b];
         const int pairs = kv_len[slot] - k + 1;
         const int rows = pairs + (n < k - 1 ? n : k - 1);
@@ -164,15 +222,19 @@ cudaError_t launch_verify_sampled(int logits_dtype, const SlotList& sl, int k, i
                                   int32_t* out_accept, int32_t* out_next, int32_t* out_kv_len, cudaStream_t st) {
     const int B = sl.n, nt = B * (k + 1), nd = B * k;
     const float inv_t = 1.0f / temperature;
-    if (logits_dtype == HIVIS_BF16) row_stats_kernel<bf16><<<nt + nd, 256, 0, st>>>(target_logits, draft_logits, nt, V, inv_t, stats);
-    else row_stats_kernel<float><<<nt + nd, 256, 0, st>>>(target_logits, draft_logits, nt, V, inv_t, stats);
+    if ((V + SV_CHUNK - 1) / SV_CHUNK > SV_MAX_CHUNKS) return cudaErrorInvalidValue;
+    const dim3 grid((unsigned)sv_pieces(V), (unsigned)(nt + nd));
+    if (logits_dtype == HIVIS_BF16) row_stats_kernel<bf16><<<grid, 256, 0, st>>>(target_logits, draft_logits, nt, V, inv_t, stats);
+    else row_stats_kernel<float><<<grid, 256, 0, st>>>(target_logits, draft_logits, nt, V, inv_t, stats);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (logits_dtype == HIVIS_BF16)
-        sampled_verify_kernel<bf16><<<B, 256, 0, st>>>(sl, k, V, inv_t, draft_ids, draft_logits, target_logits, stats, u_accept,
-                                                        u_sample, kv_len, out_accept, out_next, out_kv_len);
+        sampled_verify_kernel<bf16><<<B, SV_THREADS, 0, st>>>(sl, k, V, inv_t, draft_ids, draft_logits, target_logits, stats,
+                                                               u_accept, u_sample, kv_len, out_accept, out_next, out_kv_len);
     else
-        sampled_verify_kernel<float><<<B, 256, 0, st>>>(sl, k, V, inv_t, draft_ids, draft_logits, target_logits, stats, u_accept,
-                                                         u_sample, kv_len, out_accept, out_next, out_kv_len);
+        sampled_verify_kernel<float><<<B, SV_THREADS, 0, st>>>(sl, k, V, inv_t, draft_ids, draft_logits, target_logits, stats,
+                                                                u_accept, u_sample, kv_len, out_accept, out_next, out_kv_len);
     return cudaGetLastError();
 }
+
+int sampled_stats_entries(int max_batch, int max_k, int V) { return max_batch * (2 * max_k + 1) * sv_pieces(V); }

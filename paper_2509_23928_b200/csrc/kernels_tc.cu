@@ -301,11 +301,13 @@ struct PhaseShape {
     int nkb, ntiles;
     long long W;
 };
+// does this launch run the part of a step that arrives on barrier `seq`?
+__device__ __forceinline__ bool seq_on(const TcArgs& a, int seq) { return seq >= a.seq_first && seq <= a.seq_last; }
 __device__ __forceinline__ PhaseShape phase_shape(const TcArgs& a, int p) {
     PhaseShape s;
     s.nkb = (a.ph[p].K + TC_BK - 1) / TC_BK;
     s.ntiles = (a.ph[p].N + TC_TM - 1) / TC_TM;
-    s.W = (long long)s.nkb * s.ntiles;
+    s.W = seq_on(a, phase_seq(p)) ? (long long)s.nkb * s.ntiles : 0;      // a phase outside the launch's part has no work
     return s;
 }
 __device__ __forceinline__ long long range_lo(long long W, int c, int G) { return W * c / G; }
@@ -405,6 +407,15 @@ __device__ __forceinline__ TcAttInfo tc_att_info(const TcArgs& a, int cta, int G
             t.n[w] = u1 - u0;
         }
         t.total += t.n[w];
+    }
+    if (!seq_on(a, TC_SEQ_ATTN)) {
+#pragma unroll
+        for (int w = 0; w < TC_ATT_WARPS; ++w) {
+            t.n[w] = 0;
+            if constexpr (AttSel<GQ>::mma) t.job[w].units = 0;
+        }
+        t.total = 0;
+        t.pl.U = 0;
     }
     return t;
 }
@@ -616,7 +627,8 @@ __device__ void tc_producer_x(const TcParams& P, TcCtl* ctl, uint32_t smemB, int
 // of the step.
 __device__ void tc_gather(const TcParams& P, TcCtl* ctl, int s, int cta, int G, int etid) {
     const TcArgs& a = P.a;
-    {
+    if (!seq_on(a, TC_SEQ_GATHER)) return;
+    if (seq_on(a, TC_SEQ_ATTN)) {
         // (cos, sin) of every sequence's new position at this step, for the attention of this step; the two
         // halves of the table alternate between steps, since CTAs still in the previous attention read the other
         const int half = a.dh >> 1;
@@ -917,6 +929,7 @@ __device__ __forceinline__ void fold_partials(const TcArgs& a, float (&acc)[16],
 __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, unsigned& seg_cnt, int cta, int G,
                                   int w4, int lane) {
     const TcArgs& a = P.a;
+    if (!seq_on(a, phase_seq(p))) return;
     const int etid = w4 * 32 + lane;
     const PhaseShape sh = phase_shape(a, p);
     const long long lo = range_lo(sh.W, cta, G), hi = range_lo(sh.W, cta + 1, G);
@@ -1142,6 +1155,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
                 tc_epilogue_phase(P, ctl, s, PH_QKV, seg_cnt, cta, G, w4, lane);
             }
             // ---- attention: needs every CTA's QKV rows
+            if (seq_on(a, TC_SEQ_ATTN)) {
             if (atid == 0)
                 wait_grid(a.bar_counter, a.bar_base + (u64)G * (u64)(s * TC_BARS_PER_STEP + TC_SEQ_ATTN), ctl, a.error_flag, 7);
             if (atid == 0) phase_stamp(a, s, 20, cta, G);
@@ -1157,6 +1171,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
             if (atid == 0) {
                 phase_stamp(a, s, TC_SEQ_ATTN, cta, G);
                 red_release_add_u64(a.bar_counter, 1ull);
+            }
             }
             if (is_epi) {
                 tc_epilogue_phase(P, ctl, s, PH_O, seg_cnt, cta, G, w4, lane);

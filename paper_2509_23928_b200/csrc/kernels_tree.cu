@@ -53,6 +53,35 @@ cudaError_t launch_tree_gather(int nb, int d, const float* g_prev, const TreeBuf
     return cudaGetLastError();
 }
 
+// The level's rows in the form the tensor-core chain kernel reads them: the features as bf16 rows with their rounding
+// remainders `lo_rows` rows further down, the embedding rows of the nodes' tokens (zero rows beyond the level: the
+// tiled copy always brings all rows), and a row count of zero per column (the kernel's own attention is not used).
+__global__ void tree_operands_tc_kernel(int nb, int d, int lo_rows, const float* feat, const int* cur_id, const bf16* embed,
+                                        int vocab, bf16* feat_h, bf16* xe_h, int* pos0, int* id_flag) {
+    const int j = blockIdx.x;
+    if (j >= nb) {
+        for (int i = threadIdx.x; i < (d >> 3); i += blockDim.x)
+            ((uint4*)(xe_h + (long long)j * d))[i] = make_uint4(0u, 0u, 0u, 0u);
+        return;
+    }
+    if (threadIdx.x == 0) pos0[j] = 0;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        const float v = feat[(long long)j * d + i];
+        const bf16 hi = __float2bfloat16_rn(v);
+        feat_h[(long long)j * d + i] = hi;
+        feat_h[(long long)(j + lo_rows) * d + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
+    }
+    const int id = checked_token(cur_id[j], vocab, id_flag);
+    for (int i = threadIdx.x; i < (d >> 3); i += blockDim.x)
+        ((uint4*)(xe_h + (long long)j * d))[i] = ((const uint4*)(embed + (long long)id * d))[i];
+}
+cudaError_t launch_tree_operands_tc(int nb, int rows, int d, int lo_rows, const float* feat, const int* cur_id,
+                                    const bf16* embed, int vocab, bf16* feat_h, bf16* xe_h, int* pos0, int* id_flag,
+                                    cudaStream_t st) {
+    tree_operands_tc_kernel<<<rows, 256, 0, st>>>(nb, d, lo_rows, feat, cur_id, embed, vocab, feat_h, xe_h, pos0, id_flag);
+    return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------------------------------ K/V rows of the level
 template <typename WT>
 __global__ void tree_kv_write_kernel(const float* qkv, int ld, int qw, int Hkv, int dh, int max_len, int slot, int level,
@@ -86,7 +115,8 @@ __global__ void tree_kv_write_kernel(const float* qkv, int ld, int qw, int Hkv, 
 template <typename WT, int DH>
 __global__ void __launch_bounds__(128) tree_attn_kernel(const float* qkv, int ld, int Hq, int Hkv, int max_len, int slot,
                                                         int level, TreeBufs T, const double* inv_freq, float scale,
-                                                        const void* Kc, const void* Vc, float* attn, bf16* attn_h) {
+                                                        const void* Kc, const void* Vc, float* attn, bf16* attn_h,
+                                                        int lo_rows) {
     constexpr int EPL = DH / 32;
     __shared__ float s_m[4], s_l[4], s_acc[4][DH];
     const int h = blockIdx.x, j = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -152,14 +182,16 @@ __global__ void __launch_bounds__(128) tree_attn_kernel(const float* qkv, int ld
             const float o = A[e] / L;
             const long long oi = (long long)j * Hq * DH + h * DH + lane * EPL + e;
             attn[oi] = o;
-            attn_h[oi] = __float2bfloat16_rn(o);
+            const bf16 hi = __float2bfloat16_rn(o);
+            attn_h[oi] = hi;
+            if (lo_rows > 0) attn_h[oi + (long long)lo_rows * Hq * DH] = __float2bfloat16_rn(o - __bfloat162float(hi));
         }
     }
 }
 
 cudaError_t launch_tree_attention(int dtype, int nb, const float* qkv, int ld, int Hq, int Hkv, int dh, int max_len,
                                   int slot, int level, const TreeBufs& T, const double* inv_freq, void* Kc, void* Vc,
-                                  float* attn, bf16* attn_h, cudaStream_t st) {
+                                  float* attn, bf16* attn_h, int lo_rows, cudaStream_t st) {
     const int qw = Hq * dh;
     const float scale = 1.0f / sqrtf((float)dh);
     if (dtype == HIVIS_BF16)
@@ -170,11 +202,11 @@ cudaError_t launch_tree_attention(int dtype, int nb, const float* qkv, int ld, i
     if (e != cudaSuccess) return e;
     const dim3 grid((unsigned)Hq, (unsigned)nb);
     if (dtype == HIVIS_BF16) {
-        if (dh == 128) tree_attn_kernel<bf16, 128><<<grid, 128, 0, st>>>(qkv, ld, Hq, Hkv, max_len, slot, level, T, inv_freq, scale, Kc, Vc, attn, attn_h);
-        else tree_attn_kernel<bf16, 64><<<grid, 128, 0, st>>>(qkv, ld, Hq, Hkv, max_len, slot, level, T, inv_freq, scale, Kc, Vc, attn, attn_h);
+        if (dh == 128) tree_attn_kernel<bf16, 128><<<grid, 128, 0, st>>>(qkv, ld, Hq, Hkv, max_len, slot, level, T, inv_freq, scale, Kc, Vc, attn, attn_h, lo_rows);
+        else tree_attn_kernel<bf16, 64><<<grid, 128, 0, st>>>(qkv, ld, Hq, Hkv, max_len, slot, level, T, inv_freq, scale, Kc, Vc, attn, attn_h, lo_rows);
     } else {
-        if (dh == 128) tree_attn_kernel<float, 128><<<grid, 128, 0, st>>>(qkv, ld, Hq, Hkv, max_len, slot, level, T, inv_freq, scale, Kc, Vc, attn, attn_h);
-        else tree_attn_kernel<float, 64><<<grid, 128, 0, st>>>(qkv, ld, Hq, Hkv, max_len, slot, level, T, inv_freq, scale, Kc, Vc, attn, attn_h);
+        if (dh == 128) tree_attn_kernel<float, 128><<<grid, 128, 0, st>>>(qkv, ld, Hq, Hkv, max_len, slot, level, T, inv_freq, scale, Kc, Vc, attn, attn_h, lo_rows);
+        else tree_attn_kernel<float, 64><<<grid, 128, 0, st>>>(qkv, ld, Hq, Hkv, max_len, slot, level, T, inv_freq, scale, Kc, Vc, attn, attn_h, lo_rows);
     }
     return cudaGetLastError();
 }
