@@ -335,7 +335,8 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
              dalloc(c, &T.cand_keep, TREE_MAX_CAND) && dalloc(c, &T.cand_pos, TREE_MAX_CAND) &&
              dalloc(c, &T.cand_score, TREE_MAX_CAND) && dalloc(c, &T.kept_n, 1) && dalloc(c, &T.kept_tok, HIVIS_TREE_MAX_KEEP) &&
              dalloc(c, &T.kept_par, HIVIS_TREE_MAX_KEEP) && dalloc(c, &T.kept_store, HIVIS_TREE_MAX_KEEP) &&
-             dalloc(c, &T.row_keys, HIVIS_TREE_MAX_KEEP + 1) && dalloc(c, &c->tree_logits, (long long)TREE_MAX_TOPK * V) &&
+             dalloc(c, &T.row_keys, HIVIS_TREE_MAX_KEEP + 1) && dalloc(c, &T.piece_stats, (long long)TREE_MAX_TOPK * tree_topk_pieces((int)V)) &&
+             dalloc(c, &T.piece_keys, (long long)TREE_MAX_TOPK * tree_topk_pieces((int)V) * TREE_MAX_TOPK) && dalloc(c, &c->tree_logits, (long long)TREE_MAX_TOPK * V) &&
              dalloc(c, &c->tree_g, (long long)TREE_MAX_TOPK * d);
     }
     if (!ok) {
@@ -938,14 +939,14 @@ int hivis_draft_tree(hivis_ctx* c, int slot, int topk, int depth, int keep, cons
     const bool tc = c->tc_ok && c->opt_tc != 0;
     for (int level = 0; level < depth; ++level) {
         const int nb = level == 0 ? 1 : topk;
-        if (level > 0) CKL(c, launch_tree_gather(nb, d, c->tree_g, T, c->feat, c->feat_h, c->cur_id, st));
+        if (level > 0 && !tc) CKL(c, launch_tree_gather(nb, d, c->tree_g, T, c->feat, c->feat_h, c->cur_id, st));
         const int row = level < n_resid - 1 ? level : n_resid - 1;
         const float* rho = resid ? c->rho + (long long)row * d : nullptr;
         if (tc) {
             const int lo = tc_lo_offset(nb);
             const u64 G = (u64)c->num_sms;
-            CKL(c, launch_tree_operands_tc(nb, TC_OP_ROWS, d, lo, c->feat, c->cur_id, (const bf16*)c->embed, V, c->feat_h,
-                                           c->xe_h, c->d_pos0, c->id_flag, st));
+            CKL(c, launch_tree_operands_tc(nb, TC_OP_ROWS, d, lo, c->feat, c->cur_id, level > 0 ? c->feat : nullptr, T,
+                                           (const bf16*)c->embed, V, c->feat_h, c->xe_h, c->d_pos0, c->id_flag, st));
             TcArgs a;
             fill_tc_args(c, &a, nb, 1, lo, rho, 1, nullptr, c->tree_logits);
             a.seq_first = 0; a.seq_last = 2;                         // gather, fusion FC, QKV
@@ -972,7 +973,10 @@ int hivis_draft_tree(hivis_ctx* c, int slot, int topk, int depth, int keep, cons
             if (rc) return rc;
         }
         CKL(c, launch_tree_topk(nb, c->tree_logits, V, topk, T, st));
-        CK(c, cudaMemcpyAsync(c->tree_g, c->feat, (size_t)nb * d * sizeof(float), cudaMemcpyDeviceToDevice, st));
+        c->launches += 1;                                            // (two kernels)
+        // (the tensor-core path reads the level's outputs where the down projection left them: they are overwritten only
+        // by the next level's own down projection, after its operands were prepared)
+        if (!tc) CK(c, cudaMemcpyAsync(c->tree_g, c->feat, (size_t)nb * d * sizeof(float), cudaMemcpyDeviceToDevice, st));
         CKL(c, launch_tree_select(level, depth, nb, topk, T, st));
     }
     CKL(c, launch_tree_finalize(keep, T, out_tokens, out_parents, out_scores, out_count, st));

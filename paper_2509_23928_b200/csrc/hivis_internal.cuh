@@ -251,7 +251,11 @@ struct TreeBufs {
     // the kept nodes (the draft tree handed to the caller), for the verification
     int *kept_n, *kept_tok, *kept_par, *kept_store;
     u64* row_keys;             // [keep + 1] argmax keys of the target's rows
+    // top-k of a level's logits: per node and 4096-logit piece the (max, sum exp) and the piece's largest keys
+    float2* piece_stats;       // [TOPK][pieces]
+    u64* piece_keys;           // [TOPK][pieces][TOPK]
 };
+int tree_topk_pieces(int V);
 cudaError_t launch_tree_begin(int slot, int d, const int* kv_len, const float* pend_feat, const int* pend_id, float* feat,
                               bf16* feat_h, int* cur_id, int* d_slots, const TreeBufs& T, cudaStream_t st);
 cudaError_t launch_tree_gather(int nb, int d, const float* g_prev, const TreeBufs& T, float* feat, bf16* feat_h, int* cur_id,
@@ -260,10 +264,10 @@ cudaError_t launch_tree_attention(int dtype, int nb, const float* qkv, int ld, i
                                   int slot, int level, const TreeBufs& T, const double* inv_freq, void* Kc, void* Vc,
                                   float* attn, bf16* attn_h, int lo_rows, cudaStream_t st);
 // the level's rows as the tensor-core chain kernel reads them (`rows` = all operand rows, so that those beyond the
-// level are cleared)
+// level are cleared; g_prev non-null: the rows are gathered from the previous level's outputs on the way)
 cudaError_t launch_tree_operands_tc(int nb, int rows, int d, int lo_rows, const float* feat, const int* cur_id,
-                                    const bf16* embed, int vocab, bf16* feat_h, bf16* xe_h, int* pos0, int* id_flag,
-                                    cudaStream_t st);
+                                    const float* g_prev, const TreeBufs& T, const bf16* embed, int vocab, bf16* feat_h,
+                                    bf16* xe_h, int* pos0, int* id_flag, cudaStream_t st);
 cudaError_t launch_tree_topk(int nb, const float* logits, int V, int topk, const TreeBufs& T, cudaStream_t st);
 cudaError_t launch_tree_select(int level, int depth, int nb, int topk, const TreeBufs& T, cudaStream_t st);
 cudaError_t launch_tree_finalize(int keep, const TreeBufs& T, int32_t* out_tokens, int32_t* out_parents, float* out_scores,

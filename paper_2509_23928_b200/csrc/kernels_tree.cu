@@ -56,8 +56,11 @@ cudaError_t launch_tree_gather(int nb, int d, const float* g_prev, const TreeBuf
 // The level's rows in the form the tensor-core chain kernel reads them: the features as bf16 rows with their rounding
 // remainders `lo_rows` rows further down, the embedding rows of the nodes' tokens (zero rows beyond the level: the
 // tiled copy always brings all rows), and a row count of zero per column (the kernel's own attention is not used).
-__global__ void tree_operands_tc_kernel(int nb, int d, int lo_rows, const float* feat, const int* cur_id, const bf16* embed,
-                                        int vocab, bf16* feat_h, bf16* xe_h, int* pos0, int* id_flag) {
+// With g_prev the rows are gathered on the way (row j = the layer output of the forward that proposed node j, and node j's
+// token); without, they are taken from feat / cur_id as tree_begin left them.
+__global__ void tree_operands_tc_kernel(int nb, int d, int lo_rows, const float* feat, const int* cur_id, const float* g_prev,
+                                        TreeBufs T, const bf16* embed, int vocab, bf16* feat_h, bf16* xe_h, int* pos0,
+                                        int* id_flag) {
     const int j = blockIdx.x;
     if (j >= nb) {
         for (int i = threadIdx.x; i < (d >> 3); i += blockDim.x)
@@ -65,20 +68,22 @@ __global__ void tree_operands_tc_kernel(int nb, int d, int lo_rows, const float*
         return;
     }
     if (threadIdx.x == 0) pos0[j] = 0;
+    const float* src = g_prev ? g_prev + (long long)T.fr_pslot[j] * d : feat + (long long)j * d;
     for (int i = threadIdx.x; i < d; i += blockDim.x) {
-        const float v = feat[(long long)j * d + i];
+        const float v = src[i];
         const bf16 hi = __float2bfloat16_rn(v);
         feat_h[(long long)j * d + i] = hi;
         feat_h[(long long)(j + lo_rows) * d + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
     }
-    const int id = checked_token(cur_id[j], vocab, id_flag);
+    const int id = checked_token(g_prev ? T.fr_tok[j] : cur_id[j], vocab, id_flag);
     for (int i = threadIdx.x; i < (d >> 3); i += blockDim.x)
         ((uint4*)(xe_h + (long long)j * d))[i] = ((const uint4*)(embed + (long long)id * d))[i];
 }
 cudaError_t launch_tree_operands_tc(int nb, int rows, int d, int lo_rows, const float* feat, const int* cur_id,
-                                    const bf16* embed, int vocab, bf16* feat_h, bf16* xe_h, int* pos0, int* id_flag,
-                                    cudaStream_t st) {
-    tree_operands_tc_kernel<<<rows, 256, 0, st>>>(nb, d, lo_rows, feat, cur_id, embed, vocab, feat_h, xe_h, pos0, id_flag);
+                                    const float* g_prev, const TreeBufs& T, const bf16* embed, int vocab, bf16* feat_h,
+                                    bf16* xe_h, int* pos0, int* id_flag, cudaStream_t st) {
+    tree_operands_tc_kernel<<<rows, 256, 0, st>>>(nb, d, lo_rows, feat, cur_id, g_prev, T, embed, vocab, feat_h, xe_h, pos0,
+                                                  id_flag);
     return cudaGetLastError();
 }
 
@@ -86,16 +91,22 @@ cudaError_t launch_tree_operands_tc(int nb, int rows, int d, int lo_rows, const 
 template <typename WT>
 __global__ void tree_kv_write_kernel(const float* qkv, int ld, int qw, int Hkv, int dh, int max_len, int slot, int level,
                                      TreeBufs T, const double* inv_freq, void* Kc, void* Vc) {
+    __shared__ float2 s_cs[128];                        // (cos, sin) of the level's position: the same for every head
     const int j = blockIdx.x;
     const int P = *T.P;
     const int row = P + T.fr_store[j], pos = P + level;
     const int half = dh / 2, kvw = Hkv * dh;
+    for (int e = threadIdx.x; e < half; e += blockDim.x) {
+        float c, s;
+        rope_cs(pos, inv_freq[e], c, s);
+        s_cs[e] = make_float2(c, s);
+    }
+    __syncthreads();
     const float* k = qkv + (long long)j * ld + qw;
     const float* v = k + kvw;
     for (int i = threadIdx.x; i < Hkv * half; i += blockDim.x) {
         const int h = i / half, e = i % half;
-        float c, s;
-        rope_cs(pos, inv_freq[e], c, s);
+        const float c = s_cs[e].x, s = s_cs[e].y;
         const float x0 = k[h * dh + e], x1 = k[h * dh + e + half];
         const long long o = (((long long)slot * Hkv + h) * max_len + row) * dh;
         store_from_float<WT>(Kc, o + e, x0 * c - x1 * s);
@@ -110,8 +121,35 @@ __global__ void tree_kv_write_kernel(const float* qkv, int ld, int qw, int Hkv, 
 
 // ------------------------------------------------------------------------------------------ tree attention
 // One CTA of four warps per (query head, node).  The node attends to the prefix rows [0, P), to the rows of its
-// ancestors (the root position first) and to its own row: `level` + 1 tree rows.  Rows are dealt to the warps in
-// turn; a warp keeps a running (max, sum, accumulator) and the four are merged at the end.
+// ancestors (the root position first) and to its own row: `level` + 1 tree rows.  Blocks of 32 rows are dealt to the
+// warps in turn.  Scores: a lane takes one row of the block and the whole dot product with the query (in shared
+// memory), so no shuffle is needed; the block's probabilities then go through an online softmax, and for the weighted
+// sum of the V rows a lane owns DH/32 output elements and every row's probability is broadcast from its lane.  The four
+// warps' (max, sum, accumulator) are merged at the end.
+template <typename WT, int DH>
+__device__ __forceinline__ float tree_row_dot(const void* Kc, long long o, const float* q) {
+    float sc = 0.f;
+    if constexpr (sizeof(WT) == 2) {
+        const uint4* kp = (const uint4*)((const bf16*)Kc + o);
+#pragma unroll
+        for (int c = 0; c < DH / 8; ++c) {
+            const uint4 w = __ldg(kp + c);
+            sc = fmaf(q[8 * c + 0], bf16_lo(w.x), sc); sc = fmaf(q[8 * c + 1], bf16_hi(w.x), sc);
+            sc = fmaf(q[8 * c + 2], bf16_lo(w.y), sc); sc = fmaf(q[8 * c + 3], bf16_hi(w.y), sc);
+            sc = fmaf(q[8 * c + 4], bf16_lo(w.z), sc); sc = fmaf(q[8 * c + 5], bf16_hi(w.z), sc);
+            sc = fmaf(q[8 * c + 6], bf16_lo(w.w), sc); sc = fmaf(q[8 * c + 7], bf16_hi(w.w), sc);
+        }
+    } else {
+        const float4* kp = (const float4*)((const float*)Kc + o);
+#pragma unroll
+        for (int c = 0; c < DH / 4; ++c) {
+            const float4 w = __ldg(kp + c);
+            sc = fmaf(q[4 * c + 0], w.x, sc); sc = fmaf(q[4 * c + 1], w.y, sc);
+            sc = fmaf(q[4 * c + 2], w.z, sc); sc = fmaf(q[4 * c + 3], w.w, sc);
+        }
+    }
+    return sc;
+}
 template <typename WT, int DH>
 __global__ void __launch_bounds__(128) tree_attn_kernel(const float* qkv, int ld, int Hq, int Hkv, int max_len, int slot,
                                                         int level, TreeBufs T, const double* inv_freq, float scale,
@@ -119,45 +157,69 @@ __global__ void __launch_bounds__(128) tree_attn_kernel(const float* qkv, int ld
                                                         int lo_rows) {
     constexpr int EPL = DH / 32;
     __shared__ float s_m[4], s_l[4], s_acc[4][DH];
+    __shared__ __align__(16) float s_q[DH];
+    __shared__ float2 s_cs[DH / 2];
     const int h = blockIdx.x, j = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int P = *T.P, pos = P + level, kvh = h / (Hq / Hkv), half = DH / 2;
-    // this lane's slice of the rotated, scaled query: elements lane*EPL .. lane*EPL + EPL - 1
-    float q[EPL];
-    const float* qh = qkv + (long long)j * ld + h * DH;
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-        const int i = lane * EPL + e, f = i % half;
+    if (threadIdx.x < half) {
         float c, s;
-        rope_cs(pos, inv_freq[f], c, s);
-        const float x = qh[i], y = qh[i < half ? i + half : i - half];
-        q[e] = (i < half ? x * c - y * s : x * c + y * s) * scale;
+        rope_cs(pos, inv_freq[threadIdx.x], c, s);
+        s_cs[threadIdx.x] = make_float2(c, s);
     }
+    __syncthreads();
+    // the rotated, scaled query
+    const float* qh = qkv + (long long)j * ld + h * DH;
+    for (int i = threadIdx.x; i < DH; i += 128) {
+        const int f = i % half;
+        const float c = s_cs[f].x, s = s_cs[f].y;
+        const float x = qh[i], y = qh[i < half ? i + half : i - half];
+        s_q[i] = (i < half ? x * c - y * s : x * c + y * s) * scale;
+    }
+    __syncthreads();
     const long long base = ((long long)slot * Hkv + kvh) * max_len;
     const int nrows = P + level + 1;
     float m = -INFINITY, l = 0.f, acc[EPL];
 #pragma unroll
     for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-    for (int r = warp; r < nrows; r += 4) {
-        int row = r;
-        if (r >= P) {
+    for (int r0 = warp * 32; r0 < nrows; r0 += 128) {
+        const int r = r0 + lane;
+        const bool ok = r < nrows;
+        int row = ok ? r : 0;
+        if (ok && r >= P) {
             const int a = r - P;                                     // a-th tree row on the path: ancestors, then the node
             row = P + (a < level ? T.fr_anc[j * TREE_MAX_DEPTH + a] : T.fr_store[j]);
         }
-        const long long o = (base + row) * DH + lane * EPL;
-        float sc = 0.f, vv[EPL];
+        const float sc = ok ? tree_row_dot<WT, DH>(Kc, (base + row) * DH, s_q) : -INFINITY;
+        float bm = sc;
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) {
-            sc = fmaf(q[e], load_as_float<WT>(Kc, o + e), sc);
-            vv[e] = load_as_float<WT>(Vc, o + e);
-        }
+        for (int off = 16; off > 0; off >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, off));
+        const float mn = fmaxf(m, bm);                               // finite: the block has at least one row
+        const float corr = expf(m - mn), p = ok ? expf(sc - mn) : 0.f;
+        float ps = p;
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, off);
-        const float mn = fmaxf(m, sc);
-        const float corr = expf(m - mn), p = expf(sc - mn);
-        l = l * corr + p;
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) acc[e] = acc[e] * corr + p * vv[e];
+        for (int off = 16; off > 0; off >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, off);
+        l = l * corr + ps;
         m = mn;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) acc[e] *= corr;
+        const int nr = min(32, nrows - r0);
+#pragma unroll 4
+        for (int t = 0; t < nr; ++t) {
+            const float pj = __shfl_sync(0xffffffffu, p, t);
+            const int rowj = __shfl_sync(0xffffffffu, row, t);
+            const long long o = (base + rowj) * DH + lane * EPL;
+            if constexpr (sizeof(WT) == 2 && EPL == 4) {
+                const uint2 w = __ldg((const uint2*)((const bf16*)Vc + o));
+                acc[0] = fmaf(pj, bf16_lo(w.x), acc[0]); acc[1] = fmaf(pj, bf16_hi(w.x), acc[1]);
+                acc[2] = fmaf(pj, bf16_lo(w.y), acc[2]); acc[3] = fmaf(pj, bf16_hi(w.y), acc[3]);
+            } else if constexpr (sizeof(WT) == 2 && EPL == 2) {
+                const unsigned w = __ldg((const unsigned*)((const bf16*)Vc + o));
+                acc[0] = fmaf(pj, bf16_lo(w), acc[0]); acc[1] = fmaf(pj, bf16_hi(w), acc[1]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) acc[e] = fmaf(pj, load_as_float<WT>(Vc, o + e), acc[e]);
+            }
+        }
     }
     if (lane == 0) { s_m[warp] = m; s_l[warp] = l; }
 #pragma unroll
@@ -235,26 +297,41 @@ __device__ __forceinline__ float block_reduce_sum(float v, float* red) {
     for (int w = 0; w < 8; ++w) r += red[w];
     return r;
 }
-__global__ void __launch_bounds__(256) tree_topk_kernel(const float* logits, int V, int topk, TreeBufs T) {
+#define TREE_PIECE 4096          // logits of a node that one CTA covers (16 per thread, kept in registers)
+int tree_topk_pieces(int V) { return (V + TREE_PIECE - 1) / TREE_PIECE; }
+
+// One CTA per (piece of the row, node): the piece's maximum and sum of exp(x - max), and its `topk` largest keys, largest
+// first.  A thread keeps its 16 logits in registers and its current best key; a round takes the block's best, and only the
+// thread that owned it looks for its next one.
+__global__ void __launch_bounds__(256) tree_topk_piece_kernel(const float* logits, int V, int topk, float2* piece_stats,
+                                                              u64* piece_keys) {
     __shared__ float red[8];
     __shared__ u64 kred[8];
-    __shared__ u64 s_prev;
-    const int j = blockIdx.x;
+    const int piece = blockIdx.x, j = blockIdx.y, pieces = gridDim.x;
     const float* x = logits + (long long)j * V;
+    const int c0 = piece * TREE_PIECE;
+    u64 key[TREE_PIECE / 256];
+    float v[TREE_PIECE / 256];
     float mx = -INFINITY;
-    for (int i = threadIdx.x; i < V; i += 256) mx = fmaxf(mx, x[i]);
+#pragma unroll
+    for (int t = 0; t < TREE_PIECE / 256; ++t) {
+        const int i = c0 + t * 256 + threadIdx.x;
+        v[t] = i < V ? x[i] : -INFINITY;
+        key[t] = i < V ? pack_key(v[t], i) : 0ull;
+        mx = fmaxf(mx, v[t]);
+    }
     mx = block_reduce_max(mx, red);
     float se = 0.f;
-    for (int i = threadIdx.x; i < V; i += 256) se += expf(x[i] - mx);
+#pragma unroll
+    for (int t = 0; t < TREE_PIECE / 256; ++t) se += expf(v[t] - mx);          // exp(-inf) = 0 beyond the row
     se = block_reduce_sum(se, red);
-    const float lse = mx + logf(se);
-    u64 prev = ~0ull;
+    if (threadIdx.x == 0) piece_stats[(long long)j * pieces + piece] = make_float2(mx, se);
+    u64 mine = 0;
+#pragma unroll
+    for (int t = 0; t < TREE_PIECE / 256; ++t) mine = key[t] > mine ? key[t] : mine;
+    u64* out = piece_keys + ((long long)j * pieces + piece) * TREE_MAX_TOPK;
     for (int r = 0; r < topk; ++r) {
-        u64 best = 0;
-        for (int i = threadIdx.x; i < V; i += 256) {
-            const u64 key = pack_key(x[i], i);
-            if (key < prev && key > best) best = key;
-        }
+        u64 best = mine;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             const u64 other = __shfl_xor_sync(0xffffffffu, best, o);
@@ -263,20 +340,69 @@ __global__ void __launch_bounds__(256) tree_topk_kernel(const float* logits, int
         __syncthreads();
         if ((threadIdx.x & 31) == 0) kred[threadIdx.x >> 5] = best;
         __syncthreads();
-        if (threadIdx.x == 0) {
-            u64 b = kred[0];
-            for (int w = 1; w < 8; ++w) b = kred[w] > b ? kred[w] : b;
-            s_prev = b;
-            const int tok = b ? key_index(b) : 0;
+        best = kred[0];
+#pragma unroll
+        for (int w = 1; w < 8; ++w) best = kred[w] > best ? kred[w] : best;
+        if (threadIdx.x == 0) out[r] = best;
+        if (best != 0ull && mine == best) {         // keys are unique (they carry the token id): one owner
+            mine = 0;
+#pragma unroll
+            for (int t = 0; t < TREE_PIECE / 256; ++t) {
+                if (key[t] == best) key[t] = 0ull;
+                mine = key[t] > mine ? key[t] : mine;
+            }
+        }
+    }
+}
+
+// One warp per node: log-sum-exp of the row from its pieces, then the `topk` largest of the pieces' keys.  The packed key
+// orders by value, then by lower token id, so equal logits come out in token order.
+__global__ void __launch_bounds__(32) tree_topk_merge_kernel(const float* logits, int V, int topk, int pieces,
+                                                             const float2* piece_stats, const u64* piece_keys, TreeBufs T) {
+    const int j = blockIdx.x, lane = threadIdx.x;
+    const float* x = logits + (long long)j * V;
+    const float2* ps = piece_stats + (long long)j * pieces;
+    float mx = -INFINITY;
+    for (int c = lane; c < pieces; c += 32) mx = fmaxf(mx, ps[c].x);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float se = 0.f;
+    for (int c = lane; c < pieces; c += 32) se += ps[c].y * expf(ps[c].x - mx);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
+    const float lse = mx + logf(se);
+    // every piece's list is sorted: a lane walks the lists of its pieces from their heads
+    const u64* pk = piece_keys + (long long)j * pieces * TREE_MAX_TOPK;
+    u64 prev = ~0ull;
+    for (int r = 0; r < topk; ++r) {
+        u64 best = 0;
+        for (int c = lane; c < pieces; c += 32)
+            for (int t = 0; t < topk; ++t) {
+                const u64 key = pk[c * TREE_MAX_TOPK + t];
+                if (key < prev) {                     // the first not yet taken of this piece
+                    best = key > best ? key : best;
+                    break;
+                }
+            }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const u64 other = __shfl_xor_sync(0xffffffffu, best, o);
+            best = other > best ? other : best;
+        }
+        prev = best;
+        if (lane == 0) {
+            const int tok = best ? key_index(best) : 0;
             T.top_tok[j * TREE_MAX_TOPK + r] = tok;
             T.top_lp[j * TREE_MAX_TOPK + r] = x[tok] - lse;
         }
-        __syncthreads();
-        prev = s_prev;
     }
 }
 cudaError_t launch_tree_topk(int nb, const float* logits, int V, int topk, const TreeBufs& T, cudaStream_t st) {
-    tree_topk_kernel<<<nb, 256, 0, st>>>(logits, V, topk, T);
+    const int pieces = tree_topk_pieces(V);
+    tree_topk_piece_kernel<<<dim3((unsigned)pieces, (unsigned)nb), 256, 0, st>>>(logits, V, topk, T.piece_stats, T.piece_keys);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    tree_topk_merge_kernel<<<nb, 32, 0, st>>>(logits, V, topk, pieces, T.piece_stats, T.piece_keys, T);
     return cudaGetLastError();
 }
 
