@@ -13,6 +13,12 @@ q_j = softmax(drafter logits row j / T), x_j the token drafted at step j and the
   the draw is the inverse CDF at u_sample: the first token whose cumulative mass exceeds u_sample * total mass.
 
 The drafter's cache keeps base_len + min(n, k-1) rows, as in greedy verification.
+
+Drafting at T > 0 (the paper evaluates T = 1 besides greedy decoding, "Inference Setup"): every chained step draws its
+token from q = softmax(logits / T) instead of taking the maximum.  The draw is written as the Gumbel-max rule, which
+turns one uniform number per vocabulary entry (given as input) into an exact sample of q:
+
+  token = argmax_i ( logits_i / T - log(-log u_i) ),  u_i uniform in (0, 1), lowest index among equal values.
 """
 from __future__ import annotations
 
@@ -74,3 +80,39 @@ def verify_sampled(draft_ids, draft_logits, target_logits, temperature, u_accept
         mass = p
     nxt, gap = inverse_cdf(mass, float(u_sample))
     return n, nxt, base_len + min(n, k - 1), (margin, gap)
+
+
+def gumbel(u) -> np.ndarray:
+    """Standard Gumbel noise from uniform numbers in (0, 1): -log(-log u)."""
+    u = np.asarray(u, np.float64)
+    with np.errstate(divide="ignore"):
+        return -np.log(-np.log(u))
+
+
+def sample_gumbel(logits, temperature: float, u):
+    """The token drawn from softmax(logits / T) with the uniform numbers u [V], and the gap between the largest and the
+    second largest perturbed value (an implementation whose perturbed logits are off by less than half of it draws the
+    same token)."""
+    z = np.asarray(logits, np.float64) / float(temperature) + gumbel(u)
+    tok = int(np.argmax(z))                                  # first maximum
+    rest = np.delete(z, tok)
+    gap = float(z[tok] - rest.max()) if rest.size else np.inf
+    return tok, gap
+
+
+def draft_sampled(o, n_cached: int, pend_id: int, pend_hidden, k: int, rho, Kc, Vc, temperature: float, u):
+    """k chained draft steps of one sequence (Algorithm 1, the drafting loop; Eq. 2) in which the token of every step is
+    drawn from softmax(logits / T) by the Gumbel-max rule; u [k, V].  Step 0 runs the pending pair at row n_cached,
+    step s >= 1 the pair (layer output of step s-1, token drawn at step s-1) with residual row min(s, R-1); every step
+    appends its K/V row to Kc / Vc (modified in place).  Returns ids [k], the unperturbed logits [k, V] and the gaps [k]."""
+    lm = o._keep["lm_head"].astype(o.rt)
+    R = rho.shape[0]
+    f, tok = np.asarray(pend_hidden, o.rt), int(pend_id)
+    ids, gaps, logits = np.empty(k, np.int32), np.empty(k), np.empty((k, lm.shape[0]))
+    for s in range(k):
+        g = o.position(f, tok, rho[min(s, R - 1)], n_cached + s, Kc, Vc)
+        logits[s] = lm @ g
+        tok, gaps[s] = sample_gumbel(logits[s], temperature, u[s])
+        ids[s] = tok
+        f = g
+    return ids, logits, gaps

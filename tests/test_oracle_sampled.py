@@ -93,3 +93,59 @@ def test_low_temperature_tends_to_greedy_verification():
         dl[np.arange(k), ids] += 4.0                                  # the drafter drew its own favourites
         n, nxt, kv, _ = osmp.verify_sampled(ids, dl, tl, 1e-3, rng.random(k) * 0.98 + 0.01, rng.random(), 20)
         assert (n, nxt, kv) == o.verify(ids, tl, 20)
+
+
+# ------------------------------------------------------------------------------------------ drafting at T > 0
+def test_gumbel_max_draws_follow_the_softmax():
+    """The sampling rule against the distribution it must realise: over many seeded uniform draws the token
+    frequencies match softmax(logits / T) within four standard deviations (a Gumbel sign error, T multiplied instead of
+    divided, or noise missing on one entry fails), and two tokens give the logistic closed form."""
+    rng = np.random.default_rng(11)
+    logits = np.array([1.5, -0.3, 0.2, 2.0, -1.0, 0.7])
+    for T in (1.0, 0.5, 2.0):
+        n = 60000
+        u = rng.random((n, logits.size))
+        toks = np.argmax(logits[None, :] / T + osmp.gumbel(u), axis=1)
+        for i in range(0, n, 7919):                                  # the function itself on a sample of the draws
+            assert osmp.sample_gumbel(logits, T, u[i])[0] == toks[i]
+        freq = np.bincount(toks, minlength=logits.size) / n
+        q = osmp.softmax_t(logits, T)
+        assert np.all(np.abs(freq - q) < 4 * np.sqrt(q * (1 - q) / n) + 1e-4), (T, freq, q)
+    # V = 2: token 0 wins iff l0/T - l1/T > g1 - g0, and g1 - g0 is logistic: P(token 0) = sigmoid((l0 - l1) / T);
+    # on the boundary u1 = u0 ** exp(-(l0 - l1) / T) the two perturbed values are equal and the lower index wins
+    l0, l1, T = 0.4, -0.9, 0.8
+    u0 = 0.37
+    u1_edge = u0 ** np.exp(-(l0 - l1) / T)
+    assert osmp.sample_gumbel([l0, l1], T, [u0, u1_edge * (1 - 1e-9)])[0] == 0
+    assert osmp.sample_gumbel([l0, l1], T, [u0, min(u1_edge * (1 + 1e-6), 1 - 1e-12)])[0] == 1
+    tok, gap = osmp.sample_gumbel([l0, l1], T, [u0, u0])              # equal noise: the larger logit, gap = (l0 - l1) / T
+    assert tok == 0 and abs(gap - (l0 - l1) / T) < 1e-12
+
+
+def test_sampled_chain_with_constant_noise_is_the_greedy_chain_and_follows_its_own_tokens():
+    """Equal uniform numbers shift every logit by the same amount, so the sampled chain must coincide with the pinned
+    greedy chain (ids, logits, cache rows); with real noise every step's logits must equal the pinned chain
+    teacher-forced along the tokens that were drawn (a wrong residual row, a stale feature or token fails)."""
+    from tests.test_oracle_tree import setup, chain
+    dims, W, o, ids, hidden, rho, Kc, Vc = setup(seed=3, T=6)
+    k, T = 4, len(ids)
+    u = np.full((k, dims.vocab), 0.42)
+    K1, V1 = Kc.copy(), Vc.copy()
+    got_ids, got_logits, gaps = osmp.draft_sampled(o, T - 1, int(ids[-1]), hidden[-1], k, rho, K1, V1, 0.7, u)
+    ref, K2, V2 = chain(o, ids, hidden, rho, [], k)
+    np.testing.assert_array_equal(got_ids, ref["ids"])
+    np.testing.assert_allclose(got_logits, ref["logits"], rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(K1[:T - 1 + k], K2[:T - 1 + k], rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(V1[:T - 1 + k], V2[:T - 1 + k], rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(gaps, ref["gaps"] / 0.7, rtol=1e-9)
+
+    rng = np.random.default_rng(5)
+    u = rng.random((k, dims.vocab))
+    K1, V1 = Kc.copy(), Vc.copy()
+    s_ids, s_logits, _ = osmp.draft_sampled(o, T - 1, int(ids[-1]), hidden[-1], k, rho, K1, V1, 5.0, u)
+    assert not np.array_equal(s_ids, ref["ids"])                     # the noise moved at least one token (seeded)
+    forced, K3, V3 = chain(o, ids, hidden, rho, list(s_ids), k)
+    np.testing.assert_allclose(s_logits, forced["logits"], rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(K1[:T - 1 + k], K3[:T - 1 + k], rtol=1e-12, atol=1e-12)
+    for s in range(k):
+        assert s_ids[s] == osmp.sample_gumbel(s_logits[s], 5.0, u[s])[0]
