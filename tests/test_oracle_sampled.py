@@ -141,11 +141,12 @@ def test_sampled_chain_with_constant_noise_is_the_greedy_chain_and_follows_its_o
 
     rng = np.random.default_rng(5)
     u = rng.random((k, dims.vocab))
+    T_hot = float(np.ptp(ref["logits"][0]))                       # hot enough for the noise to matter
     K1, V1 = Kc.copy(), Vc.copy()
-    s_ids, s_logits, _ = osmp.draft_sampled(o, T - 1, int(ids[-1]), hidden[-1], k, rho, K1, V1, 5.0, u)
+    s_ids, s_logits, _ = osmp.draft_sampled(o, T - 1, int(ids[-1]), hidden[-1], k, rho, K1, V1, T_hot, u)
     assert not np.array_equal(s_ids, ref["ids"])                     # the noise moved at least one token (seeded)
     forced, K3, V3 = chain(o, ids, hidden, rho, list(s_ids), k)
     np.testing.assert_allclose(s_logits, forced["logits"], rtol=1e-12, atol=1e-12)
     np.testing.assert_allclose(K1[:T - 1 + k], K3[:T - 1 + k], rtol=1e-12, atol=1e-12)
     for s in range(k):
-        assert s_ids[s] == osmp.sample_gumbel(s_logits[s], 5.0, u[s])[0]
+        assert s_ids[s] == osmp.sample_gumbel(s_logits[s], T_hot, u[s])[0]
