@@ -596,6 +596,27 @@ def tree_and_sampling(weights: WeightCache, reps: int = 30):
                                    "us": round(us, 1), "launches": 2, "algorithmic_bytes": int(lbytes),
                                    "GBps": round(lbytes / (us * 1e-6) / 1e9, 1),
                                    "frac_of_peak": round(lbytes / (us * 1e-6) / 1e9 / peak, 4)}
+    # chained drafting with drawn tokens (T = 1) against greedy drafting, same batch
+    uni = torch.from_numpy((rng.random((B, k, V)) * (1 - 2e-6) + 1e-6).astype(np.float32)).cuda()
+    g_ms, s_ms = [], []
+    for i in range(reps + 3):
+        for sampled in (False, True):
+            for b in range(B):
+                dr.set_kv_len(b, int(lens[b]) - 1, restore_pending=True)
+            a, b_ = ev(), ev()
+            a.record()
+            if sampled:
+                dr.draft_sampled(B, k, 1.0, uni, d_resid, want_logits=False)
+            else:
+                dr.draft(B, k, d_resid, out_ids=out_ids)
+            b_.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                (s_ms if sampled else g_ms).append(a.elapsed_time(b_))
+    out["sampled_drafting"] = {"workload": wl.name, "batch": B, "k": k, "temperature": 1.0,
+                               "us_per_draft_step": round(float(np.median(s_ms)) / k * 1e3, 2),
+                               "greedy_us_per_draft_step": round(float(np.median(g_ms)) / k * 1e3, 2),
+                               "uniform_bytes_per_step": int(B * V * 4)}
     dr.status()
     dr.close()
     return out

@@ -140,6 +140,21 @@ int hivis_draft(hivis_ctx* ctx, int B, const int* seq_slots_host, int k, const v
                 int n_resid, int32_t* out_ids, const int32_t* forced_ids, float* out_logits,
                 void* stream);
 
+/* The same k chained draft steps with every step's token DRAWN from softmax(logits / temperature)
+ * instead of taken as the maximum (the paper also evaluates T = 1, "Inference Setup").  The
+ * draw is the Gumbel-max rule: token = argmax_i (logits_i / T - log(-log u_i)), lowest index
+ * among equal values, which turns one uniform number per vocabulary entry into an exact sample
+ * of that distribution; the uniform numbers are the caller's.
+ * uniforms: fp32 [B, k, vocab], device, every value in (0, 1).
+ * out_logits (nullable, fp32 [B, k, vocab]): the unperturbed LM-head outputs - the drafter's
+ * distributions that hivis_verify_sampled needs.
+ * Runs in the chain kernels only: one sequence, or up to 16 sequences of a bf16 context;
+ * anything else returns SHAPE.  Otherwise as hivis_draft (state, growth of the slots, errors;
+ * ARG also for temperature <= 0).                                                             */
+int hivis_draft_sampled(hivis_ctx* ctx, int B, const int* seq_slots_host, int k, const void* resid,
+                        int n_resid, float temperature, const float* uniforms, int32_t* out_ids,
+                        float* out_logits, void* stream);
+
 /* Batched greedy verification and KV rollback (Sec. 2.1; Algorithm 1, lines 8-9).
  * target_logits: [B, k+1, vocab] in logits_dtype (HIVIS_F32 | HIVIS_BF16); row j is the
  * target's prediction after the root token and j draft tokens.  Draft token j (0-based) is

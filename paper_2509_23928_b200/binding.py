@@ -17,7 +17,7 @@ ERRORS = {0: "OK", -1: "ARG", -2: "SHAPE", -3: "DTYPE", -4: "STATE", -5: "CAPACI
 EXPORTS = ("hivis_init", "hivis_destroy", "hivis_prefill", "hivis_draft", "hivis_verify", "hivis_reset",
            "hivis_get_kv_len", "hivis_set_kv_len", "hivis_read_kv", "hivis_debug_tap", "hivis_step_bytes",
            "hivis_launch_count", "hivis_last_error", "hivis_profile_begin", "hivis_profile_end", "hivis_set_option",
-           "hivis_status", "hivis_verify_noalloc", "hivis_read_phase_times", "hivis_draft_tree", "hivis_verify_tree", "hivis_verify_sampled")
+           "hivis_status", "hivis_verify_noalloc", "hivis_read_phase_times", "hivis_draft_tree", "hivis_verify_tree", "hivis_verify_sampled", "hivis_draft_sampled")
 HIVIS_OPT_CHAIN_KERNEL = 0
 HIVIS_OPT_TC_KERNEL = 1
 HIVIS_OPT_WAIT_LIMIT_US = 2
@@ -79,6 +79,7 @@ def _load() -> C.CDLL:
     L.hivis_profile_end.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int64)]
     L.hivis_verify_noalloc.argtypes = [i32, i32, i32, vp, vp, i32, vp, vp, vp, vp, vp]
     L.hivis_verify_sampled.argtypes = [vp, i32, ip, i32, vp, vp, vp, i32, C.c_float, vp, vp, vp, vp, vp, vp]
+    L.hivis_draft_sampled.argtypes = [vp, i32, ip, i32, vp, i32, C.c_float, vp, vp, vp, vp]
     L.hivis_draft_tree.argtypes = [vp, i32, i32, i32, i32, vp, i32, vp, vp, vp, vp, vp]
     L.hivis_verify_tree.argtypes = [vp, i32, vp, i32, vp, vp, vp, vp, vp]
     L.hivis_read_phase_times.argtypes = [vp, vp, C.c_longlong, ip, ip, vp]
@@ -144,6 +145,11 @@ def hivis_prefill(ctx, B, seq_slots, ids, hidden, cu_seqlens, start_pos=None, re
 def hivis_draft(ctx, B, seq_slots, k, resid, n_resid, out_ids, forced_ids=None, out_logits=None, stream=None):
     _check(lib.hivis_draft(ctx, int(B), _ints(seq_slots), int(k), _ptr(resid), int(n_resid), _ptr(out_ids),
                            _ptr(forced_ids), _ptr(out_logits), _stream(stream)), ctx)
+
+
+def hivis_draft_sampled(ctx, B, seq_slots, k, resid, n_resid, temperature, uniforms, out_ids, out_logits=None, stream=None):
+    _check(lib.hivis_draft_sampled(ctx, int(B), _ints(seq_slots), int(k), _ptr(resid), int(n_resid), float(temperature),
+                                   _ptr(uniforms), _ptr(out_ids), _ptr(out_logits), _stream(stream)), ctx)
 
 
 def hivis_verify(ctx, B, seq_slots, k, draft_ids, target_logits, logits_dtype, out_accept, out_next,
@@ -286,6 +292,15 @@ class Drafter:
         logits = t.empty((B, k, self.dims.vocab), dtype=t.float32, device=self.dev) if want_logits else None
         n_resid = 0 if resid is None else int(resid.shape[0])
         hivis_draft(self.ctx, B, slots, k, resid, n_resid, out_ids, forced_ids, logits)
+        return (out_ids, logits) if want_logits else out_ids
+
+    def draft_sampled(self, B, k, temperature, uniforms, resid=None, slots=None, want_logits=True):
+        """Chained drafting with every token drawn from softmax(logits / temperature); uniforms fp32 [B, k, vocab]."""
+        t = self.torch
+        out_ids = t.empty((B, k), dtype=t.int32, device=self.dev)
+        logits = t.empty((B, k, self.dims.vocab), dtype=t.float32, device=self.dev) if want_logits else None
+        hivis_draft_sampled(self.ctx, B, slots, k, resid, 0 if resid is None else int(resid.shape[0]), temperature, uniforms,
+                            out_ids, logits)
         return (out_ids, logits) if want_logits else out_ids
 
     def verify(self, draft_ids, target_logits, slots=None):

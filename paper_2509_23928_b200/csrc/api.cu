@@ -712,8 +712,10 @@ static void fill_tc_args(hivis_ctx* c, TcArgs* out, int B, int k, int lo, const 
     a.seq_first = 0; a.seq_last = 7;
 }
 
-int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const void* resid, int n_resid,
-                int32_t* out_ids, const int32_t* forced_ids, float* out_logits, void* stream) {
+// hivis_draft and hivis_draft_sampled (uniforms != nullptr: every step's token is drawn with the Gumbel-max rule)
+static int draft_impl(hivis_ctx* c, int B, const int* seq_slots_host, int k, const void* resid, int n_resid,
+                      int32_t* out_ids, const int32_t* forced_ids, float* out_logits, float inv_t, const float* uniforms,
+                      void* stream) {
     if (!c) return HIVIS_ERR_ARG;
     SlotList sl;
     int rc = check_slots(c, B, seq_slots_host, &sl);
@@ -749,6 +751,8 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
         a.slot = sl.slot[0];
         a.forced = forced_ids;
         a.logits_out = out_logits;
+        a.gumbel_u = uniforms;
+        a.inv_t = inv_t;
         a.out_ids = out_ids;
         plan_attention(c, max_rows, c->num_sms / g.n_q_heads, &a.attn_chunk, &a.attn_nsplit);
         a.bar_base = c->bar_count_host + (c->debug_skew ? (1ull << 40) : 0ull);
@@ -772,6 +776,8 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
                                               V, c->xe_h, c->id_flag, st));
         TcArgs a;
         fill_tc_args(c, &a, B, k, lo, resid ? c->rho : nullptr, resid ? n_resid : 1, forced_ids, out_logits);
+        a.gumbel_u = uniforms;
+        a.inv_t = inv_t;
         if (c->opt_phase_times) {
             CK(c, cudaMemsetAsync(c->phase_t, 0, (size_t)k * HIVIS_PHASE_EVENTS * c->num_sms * sizeof(u64), st));
             a.phase_t = c->phase_t;
@@ -791,6 +797,9 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
         c->tap_mma = true;
         return HIVIS_OK;
     }
+    if (uniforms)
+        return fail(c, HIVIS_ERR_SHAPE, "drawing the drafted tokens runs in the chain kernels only: one sequence, or up to 16 "
+                    "sequences of a bf16 context with the kernels switched on");
     CKP(c, CLS_OTHER, st, launch_draft_setup(sl, k, d, c->d_slots, c->d_pos0, c->kv_len, c->pend_feat, c->pend_id, c->feat,
                               c->feat_h, c->cur_id, c->keys, c->key_stride, st));
     const bool mma = use_mma(c, B, false);
@@ -844,6 +853,20 @@ int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const voi
     c->tap_B = B;
     c->tap_mma = mma;
     return HIVIS_OK;
+}
+
+int hivis_draft(hivis_ctx* c, int B, const int* seq_slots_host, int k, const void* resid, int n_resid,
+                int32_t* out_ids, const int32_t* forced_ids, float* out_logits, void* stream) {
+    return draft_impl(c, B, seq_slots_host, k, resid, n_resid, out_ids, forced_ids, out_logits, 0.f, nullptr, stream);
+}
+
+int hivis_draft_sampled(hivis_ctx* c, int B, const int* seq_slots_host, int k, const void* resid, int n_resid,
+                        float temperature, const float* uniforms, int32_t* out_ids, float* out_logits, void* stream) {
+    if (!c) return HIVIS_ERR_ARG;
+    if (!uniforms || misaligned(uniforms)) return fail(c, HIVIS_ERR_ARG, "uniforms is null or not 16-byte aligned");
+    if (!(temperature > 0.f)) return fail(c, HIVIS_ERR_ARG, "temperature must be positive");
+    return draft_impl(c, B, seq_slots_host, k, resid, n_resid, out_ids, nullptr, out_logits, 1.0f / temperature, uniforms,
+                      stream);
 }
 
 int hivis_verify(hivis_ctx* c, int B, const int* seq_slots_host, int k, const int32_t* draft_ids,

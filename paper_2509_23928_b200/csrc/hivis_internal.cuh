@@ -115,6 +115,8 @@ struct ChainArgs {
     u64* keys;                 // [k]
     const int* forced;         // [k], nullable
     float* logits_out;         // [k][V], nullable
+    const float* gumbel_u;     // [k][V] uniform numbers in (0, 1), nullable: the token is drawn, not the maximum
+    float inv_t;               // 1 / temperature of the draw
     int32_t* out_ids;          // [k]
     void *Kc, *Vc;
     const double* inv_freq;
@@ -174,6 +176,8 @@ struct TcArgs {
     const bf16* embed;         // [V][d]
     float *ssq1, *ssq2;        // [tiles*4][16] partial sums of squares of u / y
     float* logits_out;         // [B][k][V], nullable
+    const float* gumbel_u;     // [B][k][V] uniform numbers in (0, 1), nullable: tokens are drawn, not the maximum
+    float inv_t;               // 1 / temperature of the draw
     float* partial;            // [grid*2][16][128] split-tile partial accumulators
     int* tile_ctr;             // arrival counters of split tiles, zero between phases
     void *Kc, *Vc;
@@ -339,6 +343,10 @@ __device__ __forceinline__ u64 pack_key(float v, int idx) {
     u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
     if (v != v) u = 0u;
     return ((u64)u << 32) | (u64)(0xFFFFFFFFu - (unsigned int)idx);
+}
+// the value whose maximum is the drawn token: logit / T plus standard Gumbel noise made from a uniform number
+__device__ __forceinline__ float gumbel_perturbed(float logit, float inv_t, float u) {
+    return fmaf(logit, inv_t, -logf(-logf(u)));
 }
 __device__ __forceinline__ int key_index(u64 key) {
     return (int)(0xFFFFFFFFu - (unsigned int)(key & 0xFFFFFFFFull));

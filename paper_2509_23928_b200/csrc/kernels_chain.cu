@@ -407,7 +407,8 @@ __global__ void __launch_bounds__(CHAIN_THREADS, 1) draft_chain_kernel(const Cha
             for (int rl = tid; rl < rows; rl += CHAIN_THREADS) {
                 const float v = row_sum(PH_LM, rl);
                 if (a.logits_out) a.logits_out[(long long)s * a.V + r0 + rl] = v;
-                const u64 key = pack_key(v, r0 + rl);
+                const u64 key = a.gumbel_u ? pack_key(gumbel_perturbed(v, a.inv_t, __ldg(a.gumbel_u + (long long)s * a.V + r0 + rl)), r0 + rl)
+                                           : pack_key(v, r0 + rl);
                 best = key > best ? key : best;
             }
 #pragma unroll

@@ -791,6 +791,11 @@ __device__ __forceinline__ void epi_preload(const TcArgs& a, int p, int s, int t
             if (b < a.B) pre.add[b] = __ldcg(a.y + (long long)b * N + row);
     } else if (p == PH_QKV) {
         pre.g = a.bqkv ? __bfloat162float(a.bqkv[row]) : 0.f;
+    } else if (p == PH_LM && a.gumbel_u) {
+        // the uniform numbers of the row's token, one per sequence (the noise is added in the output stage)
+#pragma unroll
+        for (int b = 0; b < 16; ++b)
+            if (b < a.B) pre.add[b] = __ldg(a.gumbel_u + ((long long)b * a.k + s) * N + row);
     }
 }
 
@@ -863,7 +868,7 @@ __device__ void epi_output(const TcArgs& a, TcCtl* ctl, int p, int s, int tile, 
             keys[b] = 0ull;
             if (rok && b < B) {
                 if (a.logits_out) a.logits_out[((long long)b * a.k + s) * a.V + row] = val[b];
-                keys[b] = pack_key(val[b], row);
+                keys[b] = pack_key(a.gumbel_u ? gumbel_perturbed(val[b], a.inv_t, pre.add[b]) : val[b], row);
             }
         }
         // best key per sequence: over the warp, then over the four warps through shared memory, so that one

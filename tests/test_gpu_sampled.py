@@ -89,3 +89,92 @@ def test_sampled_verification_errors():
         assert (acc.cpu().numpy() == k).all() and (nxt.cpu().numpy() == 0).all()      # uniform vs uniform, u = 0
     finally:
         case.close()
+
+
+# ------------------------------------------------------------------------------------------ drafting at T > 0
+@pytest.mark.parametrize("name,temperature", [
+    ("c1_tiny_f32_b1", 1.0), ("mini_mha_b1", 0.6), ("mini_mha_b5_ragged", 1.0), ("mini_gqa_b16_ragged", 0.8),
+    ("gqa4_b5_ragged", 1.5), ("c2_llava_b1", 1.0),
+])
+def test_sampled_drafting_parity(name, temperature):
+    """hivis_draft_sampled against the oracle's chain with the same uniform numbers: ids step by step (a drawn token
+    may differ only where the two largest perturbed values lie closer than the logits' tolerance allows; the
+    sequence is then left, later steps legitimately diverge), the unperturbed logits of every compared step, the
+    appended cache rows of fully compared sequences, and on the GPU side alone: every id is the maximum of the GPU's own
+    logits / T plus the noise (fp64)."""
+    import torch
+    from tests.harness import LOGIT_RTOL, LOGIT_RTOL_F32, row_rel_err
+    wl = hi.workload(name)
+    full = name.startswith("c2_")
+    case = Case(wl)
+    try:
+        B, k, V = wl.batch, wl.k, wl.dims.vocab
+        rtol = LOGIT_RTOL if wl.dims.dtype == "bf16" else LOGIT_RTOL_F32
+        rng = np.random.default_rng(77)
+        u = (rng.random((B, k, V)) * (1 - 2e-6) + 1e-6).astype(np.float32)
+        case.gpu_prefill()
+        ids_g, logits_g = case.drafter.draft_sampled(B, k, temperature, torch.from_numpy(u).cuda(), case.d_resid)
+        torch.cuda.synchronize()
+        case.drafter.status()
+        ids_g, logits_g = ids_g.cpu().numpy(), logits_g.cpu().numpy()
+        # the GPU's draw against its own logits
+        z = logits_g.astype(np.float64) / temperature + osmp.gumbel(u.astype(np.float64))
+        top2 = np.sort(z, axis=-1)[..., -2:]
+        for b in range(B):
+            for s in range(k):
+                if top2[b, s, 1] - top2[b, s, 0] > 1e-4:
+                    assert ids_g[b, s] == int(np.argmax(z[b, s])), f"seq {b} step {s}: not the maximum of its own perturbed logits"
+        assert len(np.unique(ids_g)) > 1
+        # against the oracle
+        rho = case.oracle.fold_residuals(case.resid)
+        compared, total = 0, 0
+        for b in (range(B) if not full else [0]):
+            lo, hi_ = int(case.cu[b]), int(case.cu[b + 1])
+            T = hi_ - lo
+            Kc, Vc = case.oracle.new_cache(T + k)
+            case.oracle.prefill(case.ids[lo:hi_], case.hidden[lo:hi_], rho[0], Kc, Vc)
+            ids_o, logits_o, gaps = osmp.draft_sampled(case.oracle, T - 1, int(case.ids[hi_ - 1]), case.hidden[hi_ - 1], k, rho,
+                                                       Kc, Vc, temperature, u[b].astype(np.float64))
+            total += k
+            whole = True
+            for s in range(k):
+                err = row_rel_err(logits_g[b, s], logits_o[s])
+                assert err <= rtol, f"seq {b} step {s}: logits rel err {err}"
+                if ids_g[b, s] != ids_o[s]:
+                    allowed = 2 * rtol * np.abs(logits_o[s]).max() / temperature + 1e-4
+                    assert gaps[s] < allowed, f"seq {b} step {s}: drew {ids_g[b, s]}, oracle {ids_o[s]}, gap {gaps[s]:.2e}"
+                    whole = False
+                    break
+                compared += 1
+            if whole:
+                gk, gv = case.drafter.read_kv(b, T - 1, k)
+                np.testing.assert_allclose(gk.cpu().numpy(), Kc[T - 1:T - 1 + k], rtol=0, atol=3e-2 if wl.dims.dtype == "bf16" else 1e-4)
+                np.testing.assert_allclose(gv.cpu().numpy(), Vc[T - 1:T - 1 + k], rtol=0, atol=3e-2 if wl.dims.dtype == "bf16" else 1e-4)
+        print(f"{name}: {compared} of {total} steps compared with the oracle")
+        assert compared >= 0.6 * total
+    finally:
+        case.close()
+
+
+def test_sampled_drafting_refusals():
+    import torch
+    from paper_2509_23928_b200 import HivisError
+    wl = hi.workload("tiny_f32_b4_ragged")                     # fp32 and four sequences: no chain kernel takes it
+    case = Case(wl)
+    try:
+        B, k, V = wl.batch, wl.k, wl.dims.vocab
+        case.gpu_prefill()
+        u = torch.full((B, k, V), 0.5, device="cuda")
+        with pytest.raises(HivisError) as e:
+            case.drafter.draft_sampled(B, k, 1.0, u, case.d_resid)
+        assert e.value.code == -2
+        with pytest.raises(HivisError) as e:
+            case.drafter.draft_sampled(1, k, 0.0, u, case.d_resid)
+        assert e.value.code == -1
+        ids = case.drafter.draft_sampled(1, k, 1.0, u, case.d_resid, want_logits=False)     # one sequence works; equal noise = greedy
+        case.drafter.set_kv_len(0, int(case.lens[0]) - 1, restore_pending=True)
+        ref = case.drafter.draft(1, k, case.d_resid)
+        torch.cuda.synchronize()
+        assert (ids.cpu().numpy() == ref.cpu().numpy()).all()
+    finally:
+        case.close()
