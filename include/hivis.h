@@ -102,7 +102,7 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
 /* Waits for the device to finish and frees everything the context owns.  NULL is allowed.   */
 int hivis_destroy(hivis_ctx* ctx);
 
-/* Prefix build (Algorithm 1, lines 1-2; Eq. 1).  Appends text positions to B sequences.
+/* Prefix build (Algorithm 1, the prefix build; Eq. 1).  Appends text positions to B sequences.
  * The batch is packed: sequence b owns entries [cu_seqlens_host[b], cu_seqlens_host[b+1]) of
  * `ids` (int32) and of `hidden` ([total, d], ctx dtype), T_b >= 1 entries each.  Entry p is
  * the pair (target hidden state of text token p, id of text token p+1): the causal shift of
@@ -123,7 +123,7 @@ int hivis_prefill(hivis_ctx* ctx, int B, const int* seq_slots_host, const int32_
                   const void* hidden, const int32_t* cu_seqlens_host,
                   const int32_t* start_pos_host, const void* resid0, void* stream);
 
-/* k chained greedy draft steps for B sequences (Algorithm 1, lines 3-7; Eq. 2).  Step 0 runs
+/* k chained greedy draft steps for B sequences (Algorithm 1, the drafting loop; Eq. 2).  Step 0 runs
  * the pending pair at the next cache row; step s >= 1 runs (the layer output of step s-1, the
  * token chosen at step s-1).  Each step: fuse + residual row min(s, n_resid-1) (rows beyond
  * the trained ones reuse the last, "Training Setup"), RMSNorm, QKV, RoPE, causal attention
@@ -155,7 +155,7 @@ int hivis_draft_sampled(hivis_ctx* ctx, int B, const int* seq_slots_host, int k,
                         int n_resid, float temperature, const float* uniforms, int32_t* out_ids,
                         float* out_logits, void* stream);
 
-/* Batched greedy verification and KV rollback (Sec. 2.1; Algorithm 1, lines 8-9).
+/* Batched greedy verification and KV rollback (Sec. 2.1; Algorithm 1, the verification step).
  * target_logits: [B, k+1, vocab] in logits_dtype (HIVIS_F32 | HIVIS_BF16); row j is the
  * target's prediction after the root token and j draft tokens.  Draft token j (0-based) is
  * accepted iff it equals argmax(row j) (lowest index on ties) and all earlier ones were.
@@ -209,7 +209,7 @@ int hivis_draft_tree(hivis_ctx* ctx, int slot, int topk, int depth, int keep, co
                      void* stream);
 
 /* Greedy verification of the tree drafted last on the slot, and KV compaction (Sec. 2.1; Algorithm 1,
- * lines 8-9).  target_logits: [count + 1, vocab] in logits_dtype: row 0 is the target's prediction after
+ * the verification step).  target_logits: [count + 1, vocab] in logits_dtype: row 0 is the target's prediction after
  * the root token, row 1 + i its prediction after the path that ends in kept node i.  From the root, the
  * child that carries argmax(row of the current node) is accepted (lowest index on ties) for as long as
  * there is one.  out_accept[0] = n accepted nodes (0..depth), out_path int32 [depth] = their indices

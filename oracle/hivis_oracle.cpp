@@ -90,7 +90,7 @@ static void matvec(const float* W, const float* bias, int rows, int cols, const 
 
 extern "C" {
 
-// Semantic fusion (Algorithm 1, line 1 and line 6; Sec. 3.2):
+// Semantic fusion (Algorithm 1, the fusion of the prefix and of every drafted position; Sec. 3.2):
 //   u = fc * [f ; E[id]]  (+ rho)          rho = the projected residual r^i w, may be null
 void hvo_fuse(const hvo_dims* D, const hvo_weights* W, const real* f, int id, const real* rho,
               real* u) {
@@ -265,7 +265,7 @@ void hvo_position(const hvo_dims* D, const hvo_weights* W, const real* f, int id
     }
 }
 
-// Prefix build (Algorithm 1, line 2; Eq. 1): positions 0..T-2 carry target features and
+// Prefix build (Algorithm 1, the prefix build; Eq. 1): positions 0..T-2 carry target features and
 // the initial residual rho0; only their K/V are ever consumed by a one-layer drafter.
 // Pair T-1 is left for draft step 0.  Kc, Vc: [>= T+k-1][hkv*dh].
 void hvo_prefill(const hvo_dims* D, const hvo_weights* W, int T, const int* ids,
@@ -277,7 +277,7 @@ void hvo_prefill(const hvo_dims* D, const hvo_weights* W, int T, const int* ids,
     }
 }
 
-// Chained drafting (Algorithm 1, lines 3-7; Eq. 2).  The cache holds n_cached rows; step 0
+// Chained drafting (Algorithm 1, the drafting loop; Eq. 2).  The cache holds n_cached rows; step 0
 // consumes the pending pair (pend_hidden, pend_id) at position n_cached with residual row 0;
 // step s >= 1 consumes (g of step s-1, token chosen at step s-1) at position n_cached + s
 // with residual row min(s, R-1).  rho: [R][d] projected residuals.
@@ -309,7 +309,7 @@ void hvo_draft(const hvo_dims* D, const hvo_weights* W, int n_cached, int pend_i
 
 // The same k steps with NO cache: at every step the whole sequence (T true-feature pairs
 // followed by the self-fed pairs so far) is pushed through the layer from scratch with an
-// L x L causal mask, exactly as Algorithm 1 line 4 writes M_q(prefix, ...).  Brute force
+// L x L causal mask, exactly as the drafting loop of Algorithm 1 writes M_q(prefix, ...).  Brute force
 // for small sizes; must agree with hvo_prefill + hvo_draft.
 void hvo_draft_bruteforce(const hvo_dims* D, const hvo_weights* W, int T, const int* ids,
                           const float* hidden, int k, const real* rho, int R,
@@ -376,7 +376,7 @@ void hvo_draft_bruteforce(const hvo_dims* D, const hvo_weights* W, int T, const 
         out_ids[s] = best;
         if (out_logits) std::memcpy(out_logits + (size_t)s * V, logits.data(), sizeof(real) * V);
         if (out_g) std::memcpy(out_g + (size_t)s * d, g, sizeof(real) * d);
-        if (s + 1 < k) {   // the self-fed pair of the next step (Algorithm 1, line 6)
+        if (s + 1 < k) {   // the self-fed pair of the next step (Algorithm 1, the drafting loop)
             const int p = L;
             std::memcpy(&feat[(size_t)p * d], g, sizeof(real) * d);
             tok[p] = forced_ids ? forced_ids[s] : best;
@@ -385,7 +385,7 @@ void hvo_draft_bruteforce(const hvo_dims* D, const hvo_weights* W, int T, const 
     }
 }
 
-// Greedy verification (Sec. 2.1; Algorithm 1, lines 8-9).  Row j of logits [(k+1)][V] is the
+// Greedy verification (Sec. 2.1; Algorithm 1, the verification step).  Row j of logits [(k+1)][V] is the
 // target's prediction after the root token and j draft tokens.  Draft token j (0-based) is
 // accepted iff it equals argmax(row j) and every earlier one was accepted.  n = number
 // accepted; next = argmax(row n) (the correction, or the bonus token when n == k);

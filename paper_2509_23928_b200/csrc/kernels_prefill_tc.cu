@@ -1,4 +1,4 @@
-// Prefix build on the tensor cores (Algorithm 1, lines 1-2; Eq. 1): for every packed (hidden state, token) pair
+// Prefix build on the tensor cores (Algorithm 1, the prefix build; Eq. 1): for every packed (hidden state, token) pair
 //     u = W_fc [h ; E[id]] + rho_0,   a = gamma_1 * u / rms(u),   K = RoPE(W_k a + b_k, position),   V = W_v a + b_v
 // and K, V go to the pair's cache row.  Unlike a draft step this is a dense contraction - thousands of pairs share
 // every weight tile - so it runs as two tcgen05 GEMMs with the weights as the M operand (128 rows) and 128 pairs

@@ -41,7 +41,7 @@ def orc():
     return oracle.Oracle(dims, rand_weights(dims), "f64")
 
 
-# ------------------------------------------------------------------ fusion (Sec. 3.2; Alg. 1 line 1)
+# ------------------------------------------------------------------ fusion (Sec. 3.2; Algorithm 1, the fusion step)
 def test_fuse_equals_two_products(orc):
     d = orc.dims.d
     rng = np.random.default_rng(1)
@@ -377,7 +377,7 @@ def test_cache_rows_written_are_exactly_text_positions():
     assert written.tolist() == [True] * (T + k - 1) + [False] * 3      # n_cached == T + k - 1
 
 
-# ------------------------------------------------------------------ refresh of drafted rows (Alg. 1 line 9; Eq. 2)
+# ------------------------------------------------------------------ refresh of drafted rows (Algorithm 1, after verification; Eq. 2)
 @pytest.mark.parametrize("n_new", [1, 2, 4])
 def test_prefill_at_a_start_position_equals_a_prefill_of_the_whole_pair_list(n_new):
     """After a round the accepted tokens come back with TARGET features: every prefix position carries a target
