@@ -767,6 +767,8 @@ struct EpiPre {
     float add[16];      // per sequence: the residual stream the result is added to (FC: the step's residual row)
     float g;            // RMSNorm gain of the row (FC, O) or the QKV bias
 };
+// SMP: the launch draws its tokens (a kernel variant of its own: the greedy output stage stays as it is)
+template <bool SMP>
 __device__ __forceinline__ void epi_preload(const TcArgs& a, int p, int s, int tile, int w4, int lane, EpiPre& pre) {
     const int N = a.ph[p].N;
     const int row = tile * TC_TM + w4 * 32 + lane;
@@ -791,7 +793,7 @@ __device__ __forceinline__ void epi_preload(const TcArgs& a, int p, int s, int t
             if (b < a.B) pre.add[b] = __ldcg(a.y + (long long)b * N + row);
     } else if (p == PH_QKV) {
         pre.g = a.bqkv ? __bfloat162float(a.bqkv[row]) : 0.f;
-    } else if (p == PH_LM && a.gumbel_u) {
+    } else if (SMP && p == PH_LM) {
         // the uniform numbers of the row's token, one per sequence (the noise is added in the output stage)
 #pragma unroll
         for (int b = 0; b < 16; ++b)
@@ -799,7 +801,8 @@ __device__ __forceinline__ void epi_preload(const TcArgs& a, int p, int s, int t
     }
 }
 
-__device__ void epi_output(const TcArgs& a, TcCtl* ctl, int p, int s, int tile, const float (&v)[16], const EpiPre& pre,
+template <bool SMP>
+__device__ __forceinline__ void epi_output(const TcArgs& a, TcCtl* ctl, int p, int s, int tile, const float (&v)[16], const EpiPre& pre,
                            unsigned& lm_calls, int w4, int lane) {
     const int N = a.ph[p].N;
     const int row = tile * TC_TM + w4 * 32 + lane;
@@ -868,7 +871,7 @@ __device__ void epi_output(const TcArgs& a, TcCtl* ctl, int p, int s, int tile, 
             keys[b] = 0ull;
             if (rok && b < B) {
                 if (a.logits_out) a.logits_out[((long long)b * a.k + s) * a.V + row] = val[b];
-                keys[b] = pack_key(a.gumbel_u ? gumbel_perturbed(val[b], a.inv_t, pre.add[b]) : val[b], row);
+                keys[b] = pack_key(SMP ? gumbel_perturbed(val[b], a.inv_t, pre.add[b]) : val[b], row);
             }
         }
         // best key per sequence: over the warp, then over the four warps through shared memory, so that one
@@ -931,7 +934,9 @@ __device__ __forceinline__ void fold_partials(const TcArgs& a, float (&acc)[16],
 // first thing they did in the phase): the counter is looked at while the MMAs of the segment still run, and if
 // everybody else has arrived their partials are summed right then; once the accumulator is ready the tile is
 // finished without the store, the fence, the atomic and the loads on the critical path.
-__device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, unsigned& seg_cnt, int cta, int G,
+// (inlined at its six call sites, so that every phase gets an output stage of its own)
+template <bool SMP>
+__device__ __forceinline__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, unsigned& seg_cnt, int cta, int G,
                                   int w4, int lane) {
     const TcArgs& a = P.a;
     if (!seq_on(a, phase_seq(p))) return;
@@ -976,7 +981,7 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
         }
         const int me = cta - cf;            // this CTA's place among the contributors (big phases)
         EpiPre pre;
-        epi_preload(a, p, s, tile, w4, lane, pre);
+        epi_preload<SMP>(a, p, s, tile, w4, lane, pre);
         // ---- while the MMAs of the segment run: the early look at the arrival counter
         bool early = false;
         float others[16];
@@ -1057,7 +1062,7 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
             }
             named_sync(TC_BAR_EPI, TC_EPI_THREADS);      // last_flag may be rewritten by the next segment
         }
-        if (finish) epi_output(a, ctl, p, s, tile, v, pre, lm_calls, w4, lane);
+        if (finish) epi_output<SMP>(a, ctl, p, s, tile, v, pre, lm_calls, w4, lane);
         idx += n;
     }
     // This CTA's part of the phase is done: arrive on the grid barrier.  All arrivals are counted in one
@@ -1079,7 +1084,7 @@ __device__ void tc_epilogue_phase(const TcParams& P, TcCtl* ctl, int s, int p, u
 
 }  // namespace
 
-template <int DH, int GQ>
+template <int DH, int GQ, bool SMP>
 __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_constant__ TcParams P) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     const TcArgs& a = P.a;
@@ -1156,8 +1161,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
         for (int s = 0; s < a.k; ++s) {
             if (is_epi) {
                 tc_gather(P, ctl, s, cta, G, atid);
-                tc_epilogue_phase(P, ctl, s, PH_FC, seg_cnt, cta, G, w4, lane);
-                tc_epilogue_phase(P, ctl, s, PH_QKV, seg_cnt, cta, G, w4, lane);
+                tc_epilogue_phase<SMP>(P, ctl, s, PH_FC, seg_cnt, cta, G, w4, lane);
+                tc_epilogue_phase<SMP>(P, ctl, s, PH_QKV, seg_cnt, cta, G, w4, lane);
             }
             // ---- attention: needs every CTA's QKV rows
             if (seq_on(a, TC_SEQ_ATTN)) {
@@ -1179,10 +1184,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_chain_kernel(const __grid_co
             }
             }
             if (is_epi) {
-                tc_epilogue_phase(P, ctl, s, PH_O, seg_cnt, cta, G, w4, lane);
-                tc_epilogue_phase(P, ctl, s, PH_GU, seg_cnt, cta, G, w4, lane);
-                tc_epilogue_phase(P, ctl, s, PH_DOWN, seg_cnt, cta, G, w4, lane);
-                tc_epilogue_phase(P, ctl, s, PH_LM, seg_cnt, cta, G, w4, lane);
+                tc_epilogue_phase<SMP>(P, ctl, s, PH_O, seg_cnt, cta, G, w4, lane);
+                tc_epilogue_phase<SMP>(P, ctl, s, PH_GU, seg_cnt, cta, G, w4, lane);
+                tc_epilogue_phase<SMP>(P, ctl, s, PH_DOWN, seg_cnt, cta, G, w4, lane);
+                tc_epilogue_phase<SMP>(P, ctl, s, PH_LM, seg_cnt, cta, G, w4, lane);
             }
         }
     }
@@ -1321,7 +1326,7 @@ cudaError_t tc_build_maps(TcMaps* maps, const ChainPhase* ph, int d, int qw, int
     return encode_map(maps->m[TCM_V], Vc, cache_rows, dh, 32, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
 }
 
-template <int DH, int GQ>
+template <int DH, int GQ, bool SMP>
 static cudaError_t tc_launch_t(const TcParams& P, int grid, cudaStream_t st) {
     // the shared-memory opt-in is a per-device attribute of the function: remember it per device ordinal
     static bool attr_set[HIVIS_MAX_DEVICES] = {false};
@@ -1331,12 +1336,12 @@ static cudaError_t tc_launch_t(const TcParams& P, int grid, cudaStream_t st) {
     cudaError_t e0 = cudaGetDevice(&dev);
     if (e0 != cudaSuccess) return e0;
     if (dev < 0 || dev >= HIVIS_MAX_DEVICES || !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(tc_chain_kernel<DH, GQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(tc_chain_kernel<DH, GQ, SMP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < HIVIS_MAX_DEVICES) attr_set[dev] = true;
     }
     void* params[] = {(void*)&P};
-    return cudaLaunchCooperativeKernel((const void*)tc_chain_kernel<DH, GQ>, dim3(grid), dim3(TC_THREADS), params, smem, st);
+    return cudaLaunchCooperativeKernel((const void*)tc_chain_kernel<DH, GQ, SMP>, dim3(grid), dim3(TC_THREADS), params, smem, st);
 }
 
 cudaError_t launch_tc_chain(const TcMaps& maps, const TcArgs& a, int grid, cudaStream_t st) {
@@ -1345,6 +1350,10 @@ cudaError_t launch_tc_chain(const TcMaps& maps, const TcArgs& a, int grid, cudaS
     P.a = a;
     const int G = a.Hq / a.Hkv;
     const int gq = (G % 7 == 0) ? 7 : 1;
-    if (a.dh == 128) return gq == 7 ? tc_launch_t<128, 7>(P, grid, st) : tc_launch_t<128, 1>(P, grid, st);
-    return gq == 7 ? tc_launch_t<64, 7>(P, grid, st) : tc_launch_t<64, 1>(P, grid, st);
+    if (a.gumbel_u) {
+        if (a.dh == 128) return gq == 7 ? tc_launch_t<128, 7, true>(P, grid, st) : tc_launch_t<128, 1, true>(P, grid, st);
+        return gq == 7 ? tc_launch_t<64, 7, true>(P, grid, st) : tc_launch_t<64, 1, true>(P, grid, st);
+    }
+    if (a.dh == 128) return gq == 7 ? tc_launch_t<128, 7, false>(P, grid, st) : tc_launch_t<128, 1, false>(P, grid, st);
+    return gq == 7 ? tc_launch_t<64, 7, false>(P, grid, st) : tc_launch_t<64, 1, false>(P, grid, st);
 }

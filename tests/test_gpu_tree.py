@@ -85,6 +85,7 @@ CASES = [  # workload, sequence, topk, depth, keep
     ("mini_mha_b5_ragged", 4, 1, 6, 6),              # one branch: a chain
     ("mini_mha_b5_ragged", 2, 16, 2, 256),           # widest level, more room than candidates
     ("mini_mha_b1", 0, 3, 1, 3),                     # depth 1: the root's proposals only
+    ("c2_llava_b1", 0, 10, 6, 60),                   # full size, the configuration bench.py --tree-and-sampling times
 ]
 
 
