@@ -91,11 +91,24 @@ CASES = [  # workload, sequence, topk, depth, keep
 
 @pytest.mark.parametrize("name,b,topk,depth,keep", CASES)
 def test_tree_draft_and_verify_parity(name, b, topk, depth, keep):
+    run_tree_parity(name, b, topk, depth, keep, True)
+
+
+@pytest.mark.parametrize("name,b,topk,depth,keep", [("mini_mha_b1", 0, 10, 6, 60), ("mini_gqa_b3", 1, 8, 4, 30)])
+def test_tree_parity_with_the_per_phase_kernels(name, b, topk, depth, keep):
+    """bf16 drafters run the levels in the tensor-core chain kernel by default; with that kernel switched off the
+    per-phase kernels must build the tree to the same bar."""
+    run_tree_parity(name, b, topk, depth, keep, False)
+
+
+def run_tree_parity(name, b, topk, depth, keep, tc):
     import torch
     wl = hi.workload(name)
     case = Case(wl, max_len=int(np.diff(hi.make_prompt(wl)[2]).max()) + 1 + depth * topk + 8, max_k=16)
     try:
         f32 = wl.dims.dtype == "f32"
+        if not tc:
+            case.drafter.set_tc_kernel(False)
         case.gpu_prefill()
         tok, par, sc, n = gpu_tree(case, b, topk, depth, keep)
         case.drafter.status()
