@@ -627,6 +627,84 @@ def tree_and_sampling(weights: WeightCache, reps: int = 30):
     return out
 
 
+def draft_verify_refresh_loop(weights: WeightCache, rounds: int = 40, tc_prefill_min: int = 0):
+    """Algorithm 1 as a loop on the drafter's side, batch 16 of the headline shape: draft k tokens, verify them against a
+    toy target whose accept lengths are planted (a truncated geometric law with ratio 0.75, drawn per sequence and
+    round), then rebuild the rows of the accepted tokens from the target's "true" features (seeded noise standing in for
+    them) with hivis_prefill(start_pos) and go on with the next round.  The accept counts travel to the host every round,
+    as they do to whoever runs the target.  Reported: tokens committed per round and sequence, the time of the three calls
+    (CUDA events), and committed tokens per second of drafter-side time."""
+    import torch
+    from hivis_inputs.device import to_dev
+    from paper_2509_23928_b200 import Drafter
+    wl = hi.workload(BATCH16)
+    B, k, V, d = wl.batch, wl.k, wl.dims.vocab, wl.dims.d
+    ids, hidden, cu = hi.make_prompt(wl)
+    lens = np.diff(cu).astype(np.int64)
+    resid = hi.make_residuals(wl)
+    dr = Drafter(wl.dims, weights.get(wl), max_batch=B, max_len=int(lens.max()) + rounds * (k + 1) + 8, max_k=8)
+    if tc_prefill_min:
+        dr.set_tc_prefill(tc_prefill_min)
+    d_resid = to_dev(resid, wl.dims.dtype)
+    dr.prefill(torch.from_numpy(ids).cuda(), to_dev(hidden, wl.dims.dtype), [int(x) for x in cu], resid0=d_resid[0])
+    rng = np.random.default_rng(wl.seed + 99)
+    base_logits = to_dev(rng.standard_normal((B, k + 1, V)).astype(np.float32), wl.logits_dtype)
+    pool = to_dev(rng.standard_normal((B * (k + 1) * 4, d)).astype(np.float32), wl.dims.dtype)   # "true" features to draw from
+    pw = 0.75 ** np.arange(k + 1); pw /= pw.sum()
+    out_ids = torch.empty((B, k), dtype=torch.int32, device="cuda")
+    rows_b = torch.arange(B, device="cuda")[:, None]
+    cols_k = torch.arange(k + 1, device="cuda")[None, :]
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    t_draft, t_verify, t_refresh, committed = [], [], [], 0
+    T = lens.copy()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for r in range(rounds):
+        e0, e1, e2, e3 = ev(), ev(), ev(), ev()
+        e0.record()
+        dr.draft(B, k, d_resid, out_ids=out_ids)
+        e1.record()
+        # the toy target (not timed as drafter work, but inside the wall clock): its logits agree with the first n drafted
+        # tokens of every sequence and disagree at position n
+        n_plant = torch.from_numpy(rng.choice(k + 1, size=B, p=pw)).cuda()
+        logits = base_logits.clone()
+        idx = torch.cat([out_ids.long(), out_ids[:, -1:].long()], 1)                       # [B, k+1] (last column unused)
+        bump = torch.where(cols_k < n_plant[:, None], 12.0, torch.where(cols_k == n_plant[:, None], -12.0, 0.0))
+        bump[:, k] = 0.0
+        logits[rows_b, cols_k, idx] = (logits[rows_b, cols_k, idx].float() + bump).to(logits.dtype)
+        torch.cuda.current_stream().synchronize()
+        e1b = ev(); e1b.record()
+        acc, nxt, kv = dr.verify(out_ids, logits)
+        e2.record()
+        n = acc.cpu().numpy().astype(np.int64)                                             # the host learns the outcome
+        nx = nxt.cpu().numpy()
+        oi = out_ids.cpu().numpy()
+        new_ids = np.concatenate([np.concatenate([oi[b, :n[b]], nx[b:b + 1]]) for b in range(B)]).astype(np.int32)
+        cu_new = np.concatenate([[0], np.cumsum(n + 1)]).astype(np.int32)
+        off = int(rng.integers(0, pool.shape[0] - int(cu_new[-1])))
+        dr.prefill(torch.from_numpy(new_ids).cuda(), pool[off:off + int(cu_new[-1])], [int(x) for x in cu_new],
+                   start_pos=[int(t) for t in T], resid0=d_resid[0])
+        e3.record()
+        torch.cuda.synchronize()
+        T += n + 1
+        committed += int((n + 1).sum())
+        if r >= 3:
+            t_draft.append(e0.elapsed_time(e1)); t_verify.append(e1b.elapsed_time(e2)); t_refresh.append(e2.elapsed_time(e3))
+    wall = time.perf_counter() - t0
+    dr.status()
+    dr.close()
+    us = lambda xs: round(float(np.median(xs)) * 1e3, 1)
+    side = us(t_draft) + us(t_verify) + us(t_refresh)
+    tau = committed / (rounds * B)
+    return {"workload": wl.name, "batch": B, "k": k, "rounds": rounds, "planted_accept_law": "P(n) ~ 0.75^n, n = 0..k",
+            "tokens_per_round_and_sequence": round(tau, 3), "draft_us": us(t_draft), "verify_us": us(t_verify),
+            "refresh_us": us(t_refresh), "refresh_includes": "D2H of the outcome, host packing, H2D of the new ids",
+            "drafter_side_us_per_round": round(side, 1),
+            "committed_tokens_per_s_of_drafter_time": round(B * tau / (side * 1e-6), 1),
+            "wall_ms_per_round_with_toy_target": round(wall / rounds * 1e3, 3),
+            "tc_prefill_min_pairs": tc_prefill_min or "default"}
+
+
 def stub_replica(rank: int) -> dict:
     """Stands in for the device work when HIVIS_BENCH_STUB=1 (CPU test of the launch path only): fixed fake
     times, rank 1 slower.  The line it leads to is marked as a stub and carries no measurement."""
@@ -648,6 +726,9 @@ def main():
                     help="time the prefix build with 0 / 576 / 2048 leading (visual stand-in) positions and exit")
     ap.add_argument("--tree-and-sampling", action="store_true",
                     help="time tree drafting + tree verification (one sequence) and speculative-sampling verification (batch 16)")
+    ap.add_argument("--loop", action="store_true",
+                    help="draft -> verify -> refresh rounds at batch 16 against a toy target with planted accept lengths")
+    ap.add_argument("--tc-prefill-min", type=int, default=0, help="with --loop: smallest prefill call (pairs) on the tensor-core path")
     ap.add_argument("--phase-times", action="store_true",
                     help="print where a draft step of the tensor-core chain kernel goes (its own time stamps) and exit")
     args = ap.parse_args()
@@ -706,6 +787,9 @@ def main():
         return
     if args.tree_and_sampling:
         print(json.dumps(tree_and_sampling(weights)))
+        return
+    if args.loop:
+        print(json.dumps(draft_verify_refresh_loop(weights, tc_prefill_min=args.tc_prefill_min)))
         return
     if args.phase_times:
         print(json.dumps(phase_breakdown(hi.workload(args.workload or BATCH16), weights)))

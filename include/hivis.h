@@ -268,9 +268,11 @@ int hivis_debug_tap(hivis_ctx* ctx, int which, float* out, void* stream);
  * 3 gate/up, 4 down, 5 LM head).  The tensor-core chain kernel loads the weights of the named matrices with the
  * keep-in-L2 policy instead of streaming them through: with k chained steps in one launch a subset that fits
  * in L2 beside the KV cache is then read from HBM once per launch rather than once per step.
- * HIVIS_OPT_TC_PREFILL (default 1): with bf16 weights, a hivis_prefill call of 128 pairs or more builds the prefix
- * with two tcgen05 GEMMs over all pairs at once (weights as the M operand, 128 pairs as N); 0 = always the
- * 16-pairs-per-pass kernels, which smaller calls use in any case.  Same results up to fp32 summation order.  */
+ * HIVIS_OPT_TC_PREFILL (default 1): with bf16 weights, a hivis_prefill call of HIVIS_TC_PREFILL_MIN_PAIRS pairs or more
+ * builds the prefix with two tcgen05 GEMMs over all pairs at once (weights as the M operand, 128 pairs as N); 0 = always
+ * the 16-pairs-per-pass kernels, which smaller calls use in any case; a value n > 1 = calls of n pairs or more.
+ * Same results up to fp32 summation order.                                                                     */
+#define HIVIS_TC_PREFILL_MIN_PAIRS 17     /* more than one pass of the 16-pairs kernels: measured crossover */
 enum { HIVIS_OPT_CHAIN_KERNEL = 0, HIVIS_OPT_TC_KERNEL = 1, HIVIS_OPT_WAIT_LIMIT_US = 2, HIVIS_OPT_DEBUG_MISS_BARRIER = 3,
        HIVIS_OPT_PHASE_TIMES = 4, HIVIS_OPT_L2_KEEP = 5, HIVIS_OPT_TC_PREFILL = 6 };
 int hivis_set_option(hivis_ctx* ctx, int option, int value);

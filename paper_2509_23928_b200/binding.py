@@ -386,9 +386,10 @@ class Drafter:
         """Test aid: the grid barriers of the next draft cannot complete, so its waits run out."""
         hivis_set_option(self.ctx, HIVIS_OPT_DEBUG_MISS_BARRIER, 1)
 
-    def set_tc_prefill(self, on: bool):
-        """False: hivis_prefill always uses the 16-pairs-per-pass kernels."""
-        hivis_set_option(self.ctx, HIVIS_OPT_TC_PREFILL, 1 if on else 0)
+    def set_tc_prefill(self, on):
+        """False: hivis_prefill always uses the 16-pairs-per-pass kernels; True: the default threshold; an int n > 1:
+        calls of n pairs or more take the tensor-core path."""
+        hivis_set_option(self.ctx, HIVIS_OPT_TC_PREFILL, int(on))
 
     def set_l2_keep(self, mask: int):
         """Bit p set: the tensor-core chain kernel asks L2 to keep the weights of matrix p (0 FC .. 5 LM head)."""

@@ -52,7 +52,7 @@ struct hivis_ctx {
     int opt_tc;                   // option HIVIS_OPT_TC_KERNEL: 0 off, 1 for two or more sequences, 2 always
     bool opt_phase_times;         // option HIVIS_OPT_PHASE_TIMES
     int opt_l2_keep;              // option HIVIS_OPT_L2_KEEP: phases whose weights are asked to stay in L2
-    bool opt_tc_prefill;          // option HIVIS_OPT_TC_PREFILL
+    int opt_tc_prefill;           // option HIVIS_OPT_TC_PREFILL: 0 = never, else the smallest call (pairs) that takes the tensor-core path
     bool pf_ok;                   // the tensor-core prefill can run (bf16, shapes, buffers)
     bf16 *pf_xe, *pf_xq;          // [map_cap][d] pair-major operands of the tensor-core prefill
     float* pf_ssq;                // [ceil(d / 128)][map_cap]
@@ -274,7 +274,7 @@ int hivis_init(hivis_ctx** out, const hivis_config* cfg, const hivis_weights* w,
     c->tc_partial = nullptr;
     c->opt_phase_times = false;
     c->opt_l2_keep = 0;
-    c->opt_tc_prefill = true;
+    c->opt_tc_prefill = HIVIS_TC_PREFILL_MIN_PAIRS;
     c->pf_ok = false;
     c->pf_xe = c->pf_xq = nullptr;
     c->pf_ssq = nullptr;
@@ -638,7 +638,7 @@ int hivis_prefill(hivis_ctx* c, int B, const int* seq_slots_host, const int32_t*
     }
     CKL(c, launch_prefill_setup(c->dtype, sl, cu, start, d, ids, hidden, c->kv_len, c->pend_feat, c->pend_id,
                                 c->slot_of, c->row_of, st));
-    if (c->pf_ok && c->opt_tc_prefill && total >= 128) {
+    if (c->pf_ok && c->opt_tc_prefill > 0 && total >= c->opt_tc_prefill) {
         // many pairs: the two GEMMs of the prefix build on the tensor cores, all pairs in one pass
         PrefillTcArgs a;
         memset(&a, 0, sizeof(a));
@@ -1110,7 +1110,7 @@ int hivis_set_option(hivis_ctx* c, int option, int value) {
         return HIVIS_OK;
     }
     if (option == HIVIS_OPT_TC_PREFILL) {
-        c->opt_tc_prefill = value != 0;
+        c->opt_tc_prefill = value == 1 ? HIVIS_TC_PREFILL_MIN_PAIRS : (value < 0 ? 0 : value);
         return HIVIS_OK;
     }
     if (option == HIVIS_OPT_L2_KEEP) {

@@ -210,7 +210,7 @@ def test_nan_hidden_state_gives_token_zero_on_both_sides(name, tc):
 
 @pytest.mark.parametrize("name", ["mini_gqa_b16_ragged", "mini_mha_b5_ragged", "gqa4_b16_ragged", "wide_gqa_b16_ragged"])
 def test_tensor_core_prefill_against_oracle_and_per_pass_prefill(name):
-    """The prefix build as two tcgen05 GEMMs over all pairs (calls of 128 pairs or more) and the 16-pairs-per-pass
+    """The prefix build as two tcgen05 GEMMs over all pairs (calls of more than 16 pairs) and the 16-pairs-per-pass
     kernels: the cached K/V rows of both against the oracle's, and the draft that follows."""
     import torch
     wl = hi.workload(name)
