@@ -705,3 +705,48 @@ def test_device_waits_run_out_cleanly_and_context_recovers(name, tc):
         assert err.max() <= 2e-2
     finally:
         case.close()
+
+
+def test_small_prefill_calls_on_both_prefix_build_paths():
+    """A refresh of 24 pairs (more than one pass of the 16-pairs kernels, far fewer than a 128-pair tile) through the
+    tensor-core prefix build and through the per-pass kernels, against the oracle; a 9-pair call takes the per-pass
+    kernels whatever the option says."""
+    import torch
+    wl = hi.workload("mini_mha_b1")
+    case = Case(wl, max_len=160)
+    try:
+        o, D = case.oracle, wl.dims
+        rho = o.fold_residuals(case.resid)
+        T = int(case.lens[0])
+        rng = np.random.default_rng(5)
+        for n_new in (24, 9):
+            # the continuation repeats the pending pair (its row was never cached) and starts at its row
+            new_ids = np.concatenate([case.ids[-1:], rng.integers(0, D.vocab, n_new - 1)]).astype(np.int32)
+            new_hidden = np.concatenate([case.hidden[-1:], hi.round_to_bf16(rng.standard_normal((n_new - 1, D.d)).astype(np.float32))])
+            Kc, Vc = o.new_cache(160)
+            o.prefill(case.ids, case.hidden, rho[0], Kc, Vc)
+            o.prefill(new_ids, new_hidden, rho[0], Kc, Vc, start_pos=T - 1)
+            got = {}
+            for opt in (True, False):
+                case.drafter.set_tc_prefill(opt)
+                case.drafter.reset(0)
+                case.gpu_prefill()
+                n0 = case.drafter.launch_count()
+                case.drafter.prefill(torch.from_numpy(new_ids).cuda(), to_dev(new_hidden, "bf16"), [0, n_new], start_pos=[T - 1],
+                                     resid0=case.d_resid[0])
+                launches = case.drafter.launch_count() - n0
+                case.drafter.status()
+                rows = T - 1 + n_new - 1
+                k_g, v_g = case.drafter.read_kv(0, 0, rows)
+                torch.cuda.synchronize()
+                got[opt] = (k_g.cpu().numpy(), v_g.cpu().numpy(), launches)
+                for g, want, nm in ((got[opt][0], Kc, "K"), (got[opt][1], Vc, "V")):
+                    e = np.abs(g - want[:rows]).max() / np.abs(want[:rows]).max()
+                    assert e <= 1e-2, f"{n_new} pairs, tensor-core path {opt}: {nm} rel err {e}"
+            if n_new > 16:
+                assert got[True][2] != got[False][2]            # two different sets of launches
+            else:
+                assert got[True][2] == got[False][2]            # a single pass either way
+        case.drafter.set_tc_prefill(True)
+    finally:
+        case.close()
