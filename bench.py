@@ -148,7 +148,8 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append([c.strip() for c in line.split(",")])
 
-    def stop(self):
+    def stop(self, first_row: int = 0):
+        """Summary of the samples from row `first_row` on (the rows before it were taken during the warm-up)."""
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -157,7 +158,7 @@ class ClockSampler:
         except Exception:
             pass
         sm, mx, reasons = [], None, set()
-        for r in self.rows:
+        for r in self.rows[first_row:]:
             try:
                 sm.append(float(r[1])); mx = float(r[2])
             except Exception:
@@ -280,7 +281,13 @@ def time_workload(wl, steps: int, warmup: int, rank: int, local_rank: int, world
         sampler.start()
     for _ in range(max(warmup, 3)):
         restore(); one_step()
+    if sampler.proc is not None:
+        # nvidia-smi takes a moment to deliver its first line: keep the same load running until it does
+        t_wait = time.perf_counter()
+        while not sampler.rows and time.perf_counter() - t_wait < 2.0:
+            restore(); one_step(); torch.cuda.synchronize()
     barrier()
+    first_sample = len(sampler.rows)
     n0 = dr.launch_count()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     draft_ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
@@ -296,7 +303,18 @@ def time_workload(wl, steps: int, warmup: int, rank: int, local_rank: int, world
     step_ms = np.array([a.elapsed_time(b) for a, b in ev])
     draft_ms = np.array([ev[i][0].elapsed_time(draft_ev[i]) for i in range(steps)])
     total_ms = float(step_ms.sum())
-    clocks = sampler.stop() if (rank == 0 and not short) else None
+    clocks = None
+    if rank == 0 and not short:
+        extended = False
+        if sampler.proc is not None and len(sampler.rows) - first_sample < 3:
+            # a timed region shorter than three sampling periods: the same load goes on (untimed) until three samples exist
+            extended = True
+            t_wait = time.perf_counter()
+            while len(sampler.rows) - first_sample < 3 and time.perf_counter() - t_wait < 2.0:
+                restore(); one_step(); torch.cuda.synchronize()
+        clocks = sampler.stop(first_sample)
+        if extended:
+            clocks["note"] = "timed region shorter than three sampling periods: sampling went on under the same load"
     total_ms = max_over_ranks(total_ms, dist, "cuda")
     ok_planted = bool((acc.cpu().numpy() == planted).all())
     dr.status()                                                  # no wait ran out, no id was out of range
