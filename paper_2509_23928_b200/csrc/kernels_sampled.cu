@@ -24,12 +24,43 @@ __global__ void __launch_bounds__(256) row_stats_kernel(const void* target, cons
     const float* dr = draft + (long long)(r - n_target) * V;
     float x[SV_SPAN / 256];
     float mx = -INFINITY;
+    // 16-byte loads where the rows start on 16-byte boundaries (V a multiple of 8; a vector is then inside the row or beyond it)
+    const bool vec = (V & 7) == 0;
+    if (vec && is_t && sizeof(LT) == 2) {
+        const uint4* src = (const uint4*)((const bf16*)target + (long long)r * V + c0);
 #pragma unroll
-    for (int j = 0; j < SV_SPAN / 256; ++j) {
-        const int i = c0 + j * 256 + threadIdx.x;
-        x[j] = i < V ? (is_t ? load_as_float<LT>(tr, i) : __ldg(dr + i)) : -INFINITY;
-        mx = fmaxf(mx, x[j]);
+        for (int j = 0; j < SV_SPAN / 2048; ++j) {
+            const int vi = j * 256 + threadIdx.x;
+            if (c0 + vi * 8 < V) {
+                const uint4 w = __ldg(src + vi);
+                x[8 * j + 0] = bf16_lo(w.x); x[8 * j + 1] = bf16_hi(w.x); x[8 * j + 2] = bf16_lo(w.y); x[8 * j + 3] = bf16_hi(w.y);
+                x[8 * j + 4] = bf16_lo(w.z); x[8 * j + 5] = bf16_hi(w.z); x[8 * j + 6] = bf16_lo(w.w); x[8 * j + 7] = bf16_hi(w.w);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) x[8 * j + e] = -INFINITY;
+            }
+        }
+    } else if (vec && (!is_t || sizeof(LT) == 4)) {
+        const float4* src = (const float4*)((is_t ? (const float*)target + (long long)r * V : dr) + c0);
+#pragma unroll
+        for (int j = 0; j < SV_SPAN / 1024; ++j) {
+            const int vi = j * 256 + threadIdx.x;
+            if (c0 + vi * 4 < V) {
+                const float4 w = __ldg(src + vi);
+                x[4 * j + 0] = w.x; x[4 * j + 1] = w.y; x[4 * j + 2] = w.z; x[4 * j + 3] = w.w;
+            } else {
+                x[4 * j + 0] = x[4 * j + 1] = x[4 * j + 2] = x[4 * j + 3] = -INFINITY;
+            }
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < SV_SPAN / 256; ++j) {
+            const int i = c0 + j * 256 + threadIdx.x;
+            x[j] = i < V ? (is_t ? load_as_float<LT>(tr, i) : __ldg(dr + i)) : -INFINITY;
+        }
     }
+#pragma unroll
+    for (int j = 0; j < SV_SPAN / 256; ++j) mx = fmaxf(mx, x[j]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     if ((threadIdx.x & 31) == 0) redf[threadIdx.x >> 5] = mx;
@@ -116,6 +147,32 @@ __global__ void __launch_bounds__(SV_THREADS) sampled_verify_kernel(SlotList sl,
         const float q = expf((__ldg(dr + i) - md) * inv_t - ld);
         return fmaxf(p - q, 0.f);
     };
+    // four consecutive tokens at once (rows on 16-byte boundaries when V is a multiple of 8)
+    const bool vec = (V & 7) == 0;
+    auto mass4 = [&](int i, bool resid, float (&m)[4]) {
+        float lt4[4], ld4[4];
+        if (vec && i + 3 < V) {
+            if constexpr (sizeof(LT) == 2) {
+                const uint2 w = __ldg((const uint2*)((const bf16*)tr + i));
+                lt4[0] = bf16_lo(w.x); lt4[1] = bf16_hi(w.x); lt4[2] = bf16_lo(w.y); lt4[3] = bf16_hi(w.y);
+            } else {
+                const float4 w = __ldg((const float4*)((const float*)tr + i));
+                lt4[0] = w.x; lt4[1] = w.y; lt4[2] = w.z; lt4[3] = w.w;
+            }
+            if (resid) {
+                const float4 w = __ldg((const float4*)(dr + i));
+                ld4[0] = w.x; ld4[1] = w.y; ld4[2] = w.z; ld4[3] = w.w;
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float p = expf((lt4[e] - mt) * inv_t - lt);
+                m[e] = resid ? fmaxf(p - expf((ld4[e] - md) * inv_t - ld), 0.f) : p;
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) m[e] = i + e < V ? mass(i + e, resid) : 0.f;
+        }
+    };
     const int nchunks = (V + SV_CHUNK - 1) / SV_CHUNK;
     bool resid = n < k;
     int last_pos = -1;
@@ -126,13 +183,13 @@ __global__ void __launch_bounds__(SV_THREADS) sampled_verify_kernel(SlotList sl,
             double acc = 0.0;
 #pragma unroll
             for (int j = 0; j < SV_CHUNK / 128; ++j) {
-                float loc = 0.f;
+                float loc = 0.f, m4[4];
+                const int i0 = c * SV_CHUNK + j * 128 + lane * 4;
+                mass4(i0, resid, m4);
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const int i = c * SV_CHUNK + j * 128 + lane * 4 + e;
-                    const float m = i < V ? mass(i, resid) : 0.f;
-                    if (m > 0.f) last_pos = i;
-                    loc += m;
+                    if (m4[e] > 0.f) last_pos = i0 + e;
+                    loc += m4[e];
                 }
                 acc += (double)loc;
             }
@@ -167,13 +224,10 @@ __global__ void __launch_bounds__(SV_THREADS) sampled_verify_kernel(SlotList sl,
     {
         // the chunk that holds the wanted mass: four consecutive tokens per thread, an exclusive scan over the block
         const int c0 = s_chunk * SV_CHUNK;
-        float m[4], loc = 0.f;
+        float m[4] = {0.f, 0.f, 0.f, 0.f}, loc = 0.f;
+        if (tid < SV_CHUNK / 4) mass4(c0 + tid * 4, resid, m);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int i = c0 + tid * 4 + e;
-            m[e] = (tid < SV_CHUNK / 4 && i < V) ? mass(i, resid) : 0.f;
-            loc += m[e];
-        }
+        for (int e = 0; e < 4; ++e) loc += m[e];
         // (should rounding keep the scan below the wanted mass although the chunk sums said it is here: the chunk's
         // last token with mass)
         if (loc > 0.f) atomicMax(&s_clast, c0 + tid * 4 + (m[3] > 0.f ? 3 : m[2] > 0.f ? 2 : m[1] > 0.f ? 1 : 0));
