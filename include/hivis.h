@@ -175,10 +175,10 @@ int hivis_verify(hivis_ctx* ctx, int B, const int* seq_slots_host, int k,
  * q_j = softmax(drafter row j / T): draft token j is kept while u_accept[b, j] < min(1, p_j(x) / q_j(x));
  * n = number kept; the next token is drawn by inverse CDF at u_sample[b] from max(0, p_n - q_n) (n < k) or
  * from p_k (n = k): the first token whose cumulative mass exceeds u_sample[b] times the total mass.
- *   draft_logits fp32 [B, k, vocab]: the drafter's logits of the k steps (hivis_draft's out_logits);
+ *   draft_logits fp32 [B, k, vocab]: the drafter's logits of the k steps (out_logits of hivis_draft_sampled / hivis_draft);
  *   target_logits [B, k+1, vocab] in logits_dtype; temperature > 0;
  *   u_accept fp32 [B, k], u_sample fp32 [B]: uniform numbers in [0, 1) supplied by the caller;
- *   outputs and rollback as for hivis_verify.  Must follow a hivis_draft of the same k on the same slots.
+ *   outputs and rollback as for hivis_verify.  Must follow a draft call of the same k on the same slots.
  * Errors: ARG, DTYPE, STATE, CAPACITY, CUDA.                                                            */
 int hivis_verify_sampled(hivis_ctx* ctx, int B, const int* seq_slots_host, int k, const int32_t* draft_ids,
                          const float* draft_logits, const void* target_logits, int logits_dtype,
