@@ -178,3 +178,65 @@ def test_sampled_drafting_refusals():
         assert (ids.cpu().numpy() == ref.cpu().numpy()).all()
     finally:
         case.close()
+
+
+def test_drawn_draft_plus_sampled_verification_emit_the_target_distribution():
+    """The point of the T > 0 path, end to end on the GPU: a token drawn by hivis_draft_sampled and then accepted or
+    replaced by hivis_verify_sampled is distributed as the TARGET's softmax, whatever the drafter's distribution.
+    16 sequences x 2500 rounds with fresh uniform numbers; the target's first row is the drafter's own step-0 logits
+    with eight tokens raised by 6, so that both the acceptance and the replacement branch are taken often.  The
+    frequencies of the eight raised tokens and of "any other token" are compared with the target's probabilities
+    (computed in fp64 from the logits the GPU returned) at four standard deviations."""
+    import torch
+    wl = hi.scaled(hi.workload("mini_gqa_b16_ragged"), k=1)
+    case = Case(wl)
+    try:
+        B, V, T = wl.batch, wl.dims.vocab, 1.0
+        case.gpu_prefill()
+        _, l0 = case.gpu_draft(1)                                    # step-0 logits [B, 1, V]: independent of any draw
+        rng = np.random.default_rng(123)
+        raised = np.stack([rng.choice(V, 8, replace=False) for _ in range(B)])          # [B, 8]
+        tl = np.zeros((B, 2, V), np.float32)
+        tl[:, 0] = l0[:, 0]
+        for b in range(B):
+            tl[b, 0, raised[b]] += 6.0
+        tl[:, 1] = rng.standard_normal((B, V)).astype(np.float32)
+        p = np.stack([osmp.softmax_t(tl[b, 0], T) for b in range(B)])                   # the target's distribution [B, V]
+        q = np.stack([osmp.softmax_t(l0[b, 0], T) for b in range(B)])
+        accept_rate = float(np.mean([np.minimum(p[b], q[b]).sum() for b in range(B)]))
+        assert 0.2 < accept_rate < 0.95                              # both branches matter
+        d_tl = torch.from_numpy(tl).cuda()
+        d_raised = torch.from_numpy(raised).cuda()
+        gen = torch.Generator(device="cuda"); gen.manual_seed(9)
+        rounds = 2500
+        hits = torch.zeros((B, 8), dtype=torch.int64, device="cuda")
+        kept = torch.zeros((), dtype=torch.int64, device="cuda")
+        for _ in range(rounds):
+            case.gpu_restore()
+            u = torch.rand((B, 1, V), generator=gen, device="cuda") * (1 - 2e-6) + 1e-6
+            ids, dl = case.drafter.draft_sampled(B, 1, T, u, case.d_resid)
+            ua = torch.rand((B, 1), generator=gen, device="cuda")
+            us = torch.rand((B,), generator=gen, device="cuda")
+            acc, nxt, _ = case.drafter.verify_sampled(ids, dl, d_tl, T, ua, us)
+            first = torch.where(acc >= 1, ids[:, 0], nxt)            # the token that is emitted at the first position
+            hits += (first[:, None] == d_raised).long()
+            kept += (acc >= 1).sum()
+        torch.cuda.synchronize()
+        case.drafter.status()
+        hits = hits.cpu().numpy()
+        n = rounds
+        for b in range(B):
+            exp = p[b, raised[b]]
+            sd = np.sqrt(exp * (1 - exp) / n)
+            assert np.all(np.abs(hits[b] / n - exp) < 4 * sd + 2e-3), (b, hits[b] / n, exp)
+            other = 1.0 - hits[b].sum() / n
+            eo = 1.0 - exp.sum()
+            assert abs(other - eo) < 4 * np.sqrt(eo * (1 - eo) / n) + 2e-3
+        # over all sequences: tighter
+        tot = hits.sum(0) / (n * B)
+        np.testing.assert_allclose(tot, p[np.arange(B)[:, None], raised].mean(0), atol=4e-3)
+        got_rate = int(kept.item()) / (n * B)
+        assert abs(got_rate - accept_rate) < 0.02, (got_rate, accept_rate)
+        print(f"acceptance rate {got_rate:.3f} (expected {accept_rate:.3f})")
+    finally:
+        case.close()
