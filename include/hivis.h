@@ -233,6 +233,11 @@ int hivis_get_kv_len(hivis_ctx* ctx, int slot, int* n_rows_host, int* pending_ho
  * benchmark return to the state right after prefill between timed repetitions.               */
 int hivis_set_kv_len(hivis_ctx* ctx, int slot, int n_rows, int restore_pending, void* stream);
 
+/* The same for B slots in one launch: slots_host[b] (NULL = slots 0..B-1, each at most once) gets
+ * n_rows_host[b] rows.  Errors: ARG, STATE, CAPACITY as above; nothing is changed when one is returned. */
+int hivis_set_kv_len_batch(hivis_ctx* ctx, int B, const int* slots_host, const int* n_rows_host,
+                           int restore_pending, void* stream);
+
 /* Debug: copy rows [row0, row0+n) of the slot's K and V cache, widened to fp32, into
  * out_k / out_v, each [n, n_kv_heads*head_dim].                                               */
 int hivis_read_kv(hivis_ctx* ctx, int slot, int row0, int n, float* out_k, float* out_v,

@@ -17,7 +17,8 @@ ERRORS = {0: "OK", -1: "ARG", -2: "SHAPE", -3: "DTYPE", -4: "STATE", -5: "CAPACI
 EXPORTS = ("hivis_init", "hivis_destroy", "hivis_prefill", "hivis_draft", "hivis_verify", "hivis_reset",
            "hivis_get_kv_len", "hivis_set_kv_len", "hivis_read_kv", "hivis_debug_tap", "hivis_step_bytes",
            "hivis_launch_count", "hivis_last_error", "hivis_profile_begin", "hivis_profile_end", "hivis_set_option",
-           "hivis_status", "hivis_verify_noalloc", "hivis_read_phase_times", "hivis_draft_tree", "hivis_verify_tree", "hivis_verify_sampled", "hivis_draft_sampled")
+           "hivis_status", "hivis_verify_noalloc", "hivis_read_phase_times", "hivis_draft_tree", "hivis_verify_tree", "hivis_verify_sampled", "hivis_draft_sampled",
+           "hivis_set_kv_len_batch")
 HIVIS_OPT_CHAIN_KERNEL = 0
 HIVIS_OPT_TC_KERNEL = 1
 HIVIS_OPT_WAIT_LIMIT_US = 2
@@ -67,6 +68,7 @@ def _load() -> C.CDLL:
     L.hivis_reset.argtypes = [vp, i32, vp]
     L.hivis_get_kv_len.argtypes = [vp, i32, ip, ip, vp]
     L.hivis_set_kv_len.argtypes = [vp, i32, i32, i32, vp]
+    L.hivis_set_kv_len_batch.argtypes = [vp, i32, ip, ip, i32, vp]
     L.hivis_read_kv.argtypes = [vp, i32, i32, i32, vp, vp, vp]
     L.hivis_debug_tap.argtypes = [vp, i32, vp, vp]
     L.hivis_step_bytes.argtypes = [vp, i32, ip]
@@ -198,6 +200,11 @@ def hivis_get_kv_len(ctx, slot, stream=None):
 
 def hivis_set_kv_len(ctx, slot, n_rows, restore_pending=False, stream=None):
     _check(lib.hivis_set_kv_len(ctx, int(slot), int(n_rows), int(bool(restore_pending)), _stream(stream)), ctx)
+
+
+def hivis_set_kv_len_batch(ctx, B, seq_slots, n_rows, restore_pending=False, stream=None):
+    _check(lib.hivis_set_kv_len_batch(ctx, int(B), _ints(seq_slots), _ints(n_rows), 1 if restore_pending else 0,
+                                      _stream(stream)), ctx)
 
 
 def hivis_read_kv(ctx, slot, row0, n, out_k, out_v, stream=None):
@@ -351,6 +358,9 @@ class Drafter:
 
     def set_kv_len(self, slot, n_rows, restore_pending=False):
         hivis_set_kv_len(self.ctx, slot, n_rows, restore_pending)
+
+    def set_kv_len_batch(self, n_rows, slots=None, restore_pending=False):
+        hivis_set_kv_len_batch(self.ctx, len(n_rows), slots, [int(x) for x in n_rows], restore_pending)
 
     def reset(self, slot):
         hivis_reset(self.ctx, slot)

@@ -1075,6 +1075,32 @@ int hivis_set_kv_len(hivis_ctx* c, int slot, int n_rows, int restore_pending, vo
     return HIVIS_OK;
 }
 
+int hivis_set_kv_len_batch(hivis_ctx* c, int B, const int* slots_host, const int* n_rows_host, int restore_pending,
+                           void* stream) {
+    if (!c) return HIVIS_ERR_ARG;
+    if (!n_rows_host) return fail(c, HIVIS_ERR_ARG, "n_rows_host is null");
+    SlotList sl;
+    int rc = check_slots(c, B, slots_host, &sl);
+    if (rc) return rc;
+    CuSeqlens rows;
+    for (int b = 0; b < B; ++b) {
+        if (n_rows_host[b] < 0 || n_rows_host[b] > c->cfg.max_len)
+            return fail(c, HIVIS_ERR_CAPACITY, "n_rows %d outside [0,%d]", n_rows_host[b], c->cfg.max_len);
+        if (restore_pending && !c->have_pair[sl.slot[b]]) return fail(c, HIVIS_ERR_STATE, "slot %d never held a pair", sl.slot[b]);
+        rows.v[b] = n_rows_host[b];
+    }
+    CKL(c, launch_set_rows(sl, rows, c->kv_len, (cudaStream_t)stream));
+    for (int b = 0; b < B; ++b) {
+        const int s = sl.slot[b];
+        c->kv_upper[s] = n_rows_host[b];
+        c->kv_exact[s] = true;
+        if (restore_pending) c->pending[s] = true;
+        c->last_k[s] = 0;
+        c->tree_depth[s] = 0;
+    }
+    return HIVIS_OK;
+}
+
 int hivis_read_kv(hivis_ctx* c, int slot, int row0, int n, float* out_k, float* out_v, void* stream) {
     if (!c) return HIVIS_ERR_ARG;
     if (slot < 0 || slot >= c->cfg.max_batch) return fail(c, HIVIS_ERR_ARG, "slot %d out of range", slot);

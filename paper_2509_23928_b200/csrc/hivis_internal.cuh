@@ -324,6 +324,8 @@ cudaError_t launch_verify_sampled(int logits_dtype, const SlotList& sl, int k, i
                                   int32_t* out_accept, int32_t* out_next, int32_t* out_kv_len, cudaStream_t st);
 
 cudaError_t launch_set_int(int* p, int v, cudaStream_t st);
+// kv_len[sl.slot[b]] = rows.v[b] for b < sl.n
+cudaError_t launch_set_rows(const SlotList& sl, const CuSeqlens& rows, int* kv_len, cudaStream_t st);
 
 // weight re-layout at init
 cudaError_t launch_copy_rows(const void* src, void* dst, long long rows, long long row_bytes,

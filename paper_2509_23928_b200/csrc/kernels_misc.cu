@@ -275,6 +275,13 @@ cudaError_t launch_verify(int logits_dtype, const SlotList& sl, int k, int V, co
 }
 
 __global__ void set_int_kernel(int* p, int v) { *p = v; }
+__global__ void set_rows_kernel(SlotList sl, CuSeqlens rows, int* kv_len) {
+    if ((int)threadIdx.x < sl.n) kv_len[sl.slot[threadIdx.x]] = rows.v[threadIdx.x];
+}
+cudaError_t launch_set_rows(const SlotList& sl, const CuSeqlens& rows, int* kv_len, cudaStream_t st) {
+    set_rows_kernel<<<1, HIVIS_MAX_BATCH, 0, st>>>(sl, rows, kv_len);
+    return cudaGetLastError();
+}
 cudaError_t launch_set_int(int* p, int v, cudaStream_t st) {
     set_int_kernel<<<1, 1, 0, st>>>(p, v);
     return cudaGetLastError();

@@ -45,8 +45,7 @@ class Case:
         self.drafter.prefill(self.d_ids, self.d_hidden, [int(x) for x in self.cu], resid0=self.d_resid[0])
 
     def gpu_restore(self):
-        for b in range(self.wl.batch):
-            self.drafter.set_kv_len(b, int(self.lens[b]) - 1, restore_pending=True)
+        self.drafter.set_kv_len_batch([int(l) - 1 for l in self.lens], restore_pending=True)
 
     def gpu_draft(self, k=None, forced=None, want_logits=True):
         t = self.torch

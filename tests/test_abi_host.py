@@ -66,6 +66,8 @@ def test_null_context_is_an_argument_error():
     assert lib.hivis_verify(None, 1, None, 1, None, None, 0, None, None, None, None) == -1
     assert lib.hivis_prefill(None, 1, None, None, None, None, None, None, None) == -1
     assert lib.hivis_step_bytes(None, 0, None) == 0
+    assert lib.hivis_draft_sampled(None, 1, None, 1, None, 0, 1.0, None, None, None, None) == -1
+    assert lib.hivis_set_kv_len_batch(None, 1, None, None, 0, None) == -1
 
 
 def test_product_package_does_not_import_the_oracle():

@@ -549,6 +549,9 @@ def test_host_side_errors_do_not_launch():
         with pytest.raises(HivisError) as e:                     # duplicate slot / too many sequences
             dr.prefill(case.d_ids, case.d_hidden, [0, 16, 32], resid0=None)
         assert e.value.code == -5
+        with pytest.raises(HivisError) as e:                     # batched row counts: one out of range, nothing changes
+            dr.set_kv_len_batch([10 ** 6])
+        assert e.value.code == -5
         with pytest.raises(HivisError) as e:                     # misaligned pointer
             dr.prefill(case.d_ids[1:], case.d_hidden, [0, 31])
         assert e.value.code == -1
